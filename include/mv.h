@@ -1,0 +1,167 @@
+/*
+ * mv.h — C ABI of the B200 batched RGB-D renderer for voxel-grid worlds.
+ *
+ * The library implements the Render half of the paper's batched simulation step
+ * (Section 3.2, Eq. 2: O(t+1) = Render(S(t+1))) for N environments x M agents in one call
+ * (Section 3.2; Appendix A.1: one step returns N x M observations).  The state of one
+ * environment is the discretised world of Section 3.1 (a voxel grid) plus the movable
+ * entities of Section 3.2 (interactive objects and agent bodies) as axis-aligned boxes, plus
+ * one camera per agent.  Observations are W x H RGB frames (Appendix A.2: 128 x 72 x 3) with
+ * an added float depth channel.  The paper renders with a batched rasteriser; this library
+ * casts one primary ray per pixel centre, which yields the same visible surface.
+ *
+ * Geometry conventions (the paper leaves them open):
+ *   - y is up.  Voxel (i,j,k) is the unit cube [i,i+1] x [j,j+1] x [k,k+1]; the grid starts
+ *     at the world origin.  Input grids are uint8 material ids, 0 = empty, laid out
+ *     [env][j (y)][k (z)][i (x)] with x fastest.
+ *   - yaw 0 looks along +z and grows toward +x; pitch > 0 looks up; image row 0 is the top.
+ *   - depth is planar: distance along the view axis, in voxel units.  A pixel that hits
+ *     nothing gets sky_rgb and miss_depth.  A camera inside a solid gets depth 0 and the
+ *     ambient-only colour of that solid.
+ *   - colour = palette[env][material] * (ambient + (1-ambient) * max(0, n . L)), L the unit
+ *     direction to the light, n the face normal, rounded half up to uint8 (evaluated in
+ *     double when palettes are uploaded).
+ *   - observation index = env * agents_per_env + agent.
+ *
+ * Memory and ownership.  Every pointer named d_* is DEVICE memory owned by the caller; the
+ * library reads or writes it only inside the stream work the call enqueues and never keeps
+ * it.  Every pointer named h_* is HOST memory owned by the caller.  Output buffers must be
+ * 16-byte aligned.  The library owns only what mv_create_batch allocates; mv_destroy frees it.
+ *
+ * Asynchrony.  All device work is enqueued on the cuda_stream argument (a cudaStream_t cast to
+ * void*, NULL = the legacy default stream).  Calls do not synchronise, except mv_query_status,
+ * mv_step_host and mv_destroy.
+ *
+ * Errors.  Every call returns MV_OK (0) or a negative mv_status.  Nothing throws or aborts.
+ * Bad data (material id >= palette_size, box count > max_boxes, non-finite camera) never causes
+ * an out-of-bounds access: ids and counts are clamped, a non-finite camera renders a sky frame,
+ * and a sticky bit is set in the device status word (see mv_query_status).
+ */
+#ifndef MV_H
+#define MV_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum mv_status {
+    MV_OK = 0,
+    MV_ERR_INVALID_ARG = -1,     /* null pointer, size out of range, bad descriptor */
+    MV_ERR_OUT_OF_MEMORY = -2,   /* device or host allocation failed */
+    MV_ERR_CUDA = -3,            /* a CUDA runtime call failed */
+    MV_ERR_NOT_READY = -4,       /* render before every env has a grid and palette, or before cameras */
+    MV_ERR_DEVICE_TIMEOUT = -5,  /* a bounded device-side wait gave up (reported by mv_query_status) */
+    MV_ERR_UNSUPPORTED = -6      /* configuration exceeds a documented limit */
+} mv_status;
+
+/* Sticky data-error bits returned (as a positive value) by mv_query_status. */
+#define MV_FLAG_MATERIAL_CLAMPED 0x1u   /* a voxel or box material id was >= palette_size */
+#define MV_FLAG_BOX_COUNT_CLAMPED 0x2u  /* a box count was > max_boxes or negative */
+#define MV_FLAG_BAD_CAMERA 0x4u         /* a camera had a non-finite component */
+#define MV_FLAG_DEVICE_TIMEOUT 0x8u     /* a staging wait in the render kernel timed out */
+
+typedef struct mv_batch mv_batch;       /* opaque; owned by the library */
+
+/* A movable entity of Section 3.2 reduced to an axis-aligned box.  32 bytes.
+ * A box with min >= max on any axis is ignored. */
+typedef struct mv_box {
+    float min[3];
+    float max[3];
+    uint32_t material;                  /* palette index */
+    uint32_t pad;
+} mv_box;
+
+/* One agent camera.  24 bytes.  self_box is the index (within the env's box list) of the
+ * agent's own body, which this camera does not see; -1 for none. */
+typedef struct mv_camera {
+    float pos[3];
+    float yaw, pitch;                   /* radians */
+    int32_t self_box;
+} mv_camera;
+
+typedef struct mv_batch_desc {
+    int32_t num_envs;                   /* N >= 1 */
+    int32_t agents_per_env;             /* M >= 1 */
+    int32_t grid_x, grid_y, grid_z;     /* voxels per axis; each a multiple of 4, 4..1024;
+                                           grid_x*grid_y*grid_z/8 bytes must fit the SM's
+                                           shared memory (about 200 KiB: 1.6 M voxels) */
+    int32_t max_boxes;                  /* per env, agent bodies included; 0..256 */
+    int32_t width, height;              /* pixels; width a multiple of 8, height of 4; <= 4096 */
+    int32_t palette_size;               /* 1..256 entries per env */
+    float hfov_rad;                     /* horizontal field of view, (0, pi) */
+    float light_dir[3];                 /* direction TO the light; any non-zero length */
+    float ambient;                      /* [0, 1] */
+    uint8_t sky_rgb[3];
+    uint8_t pad;
+    float miss_depth;
+    int32_t device;                     /* CUDA device ordinal */
+} mv_batch_desc;
+
+/* Allocate the device-resident world store, camera table and status word for a batch
+ * (paper Section 3.2: one instance hosts N environments with M agents each).
+ * desc: HOST pointer.  out: HOST pointer receiving the handle.
+ * Errors: INVALID_ARG (null, out-of-range field), UNSUPPORTED (grid too large for shared
+ * memory), OUT_OF_MEMORY, CUDA. */
+int mv_create_batch(const mv_batch_desc *desc, mv_batch **out);
+
+/* Upload world state for envs [env_begin, env_begin+env_count) (paper Section 3.3: geometry
+ * is prepared once per episode; Section 3.1: objects move every step, hence any of the array
+ * arguments may be NULL meaning "keep what was uploaded before").
+ *   d_grid      DEVICE uint8 [env_count][grid_y][grid_z][grid_x]; packed on the device into a
+ *               1-bit occupancy grid plus a material store.
+ *   d_boxes     DEVICE mv_box [env_count][max_boxes]
+ *   d_box_count DEVICE int32 [env_count]; required when d_boxes is given
+ *   d_palette   DEVICE uint8 [env_count][palette_size][3]; the per-env shaded colour table
+ *               is rebuilt from it on the device
+ * Errors: INVALID_ARG (range, d_boxes without d_box_count), CUDA. */
+int mv_upload_worlds(mv_batch *batch, int env_begin, int env_count, const uint8_t *d_grid,
+                     const mv_box *d_boxes, const int32_t *d_box_count, const uint8_t *d_palette,
+                     void *cuda_stream);
+
+/* Set all cameras (paper Section 3.2: cameras are part of the state; Appendix A.1: N x M
+ * observations per step) and build each one's ray basis on the device.
+ *   d_cams DEVICE mv_camera [num_envs*agents_per_env]
+ * Errors: INVALID_ARG, CUDA. */
+int mv_set_cameras(mv_batch *batch, const mv_camera *d_cams, void *cuda_stream);
+
+/* Render every observation of the batch in one launch (paper Section 3.2, Eq. 2; "a single
+ * request to the GPU to render all the observations").
+ *   d_rgb   DEVICE uint8 [num_obs][height][width][3]
+ *   d_depth DEVICE float [num_obs][height][width]
+ * Errors: INVALID_ARG, NOT_READY (some env has no grid/palette yet, or no cameras), CUDA. */
+int mv_render_batch(mv_batch *batch, uint8_t *d_rgb, float *d_depth, void *cuda_stream);
+
+/* One whole step from HOST memory (paper Section 3.2: by default the rendered frames are
+ * transferred to CPU memory): copies cameras (and, if given, this step's boxes) host->device,
+ * builds ray bases, renders, and copies rgb and depth device->host, overlapping the copies with
+ * rendering chunk by chunk.  Synchronous: on return the host buffers hold the frames.
+ *   h_cams      HOST mv_camera [num_obs]
+ *   h_boxes     HOST mv_box [num_envs][max_boxes] or NULL (keep)
+ *   h_box_count HOST int32 [num_envs]; required when h_boxes is given
+ *   h_rgb, h_depth HOST outputs, same shapes as mv_render_batch; page-locked memory is
+ *               needed for the copies to overlap
+ * The first call allocates device-side frame buffers of the batch's full output size.
+ * Errors: as the calls it is made of. */
+int mv_step_host(mv_batch *batch, const mv_camera *h_cams, const mv_box *h_boxes,
+                 const int32_t *h_box_count, uint8_t *h_rgb, float *h_depth, void *cuda_stream);
+
+/* Synchronise the stream and return the device status word: a negative mv_status if a CUDA
+ * error or device timeout occurred, else the OR of the MV_FLAG_* bits seen so far (0 = clean).
+ * clear != 0 resets the sticky bits. */
+int mv_query_status(mv_batch *batch, int clear, void *cuda_stream);
+
+/* Number of kernels of this library launched on behalf of `batch` so far (host counter). */
+int64_t mv_launch_count(const mv_batch *batch);
+
+/* Free everything mv_create_batch allocated (synchronises the device). NULL is accepted. */
+int mv_destroy(mv_batch *batch);
+
+/* Static, never-freed description of a status code. */
+const char *mv_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MV_H */

@@ -52,9 +52,11 @@ def make_desc(grid_shape, max_boxes, width, height, palette_size, hfov=np.pi / 2
     d = Desc()
     d.gx, d.gy, d.gz, d.max_boxes = gx, gy, gz, max_boxes
     d.width, d.height, d.palette_size = width, height, palette_size
-    d.hfov = float(hfov)
-    d.light_dir = (C.c_double * 3)(*[float(x) for x in light_dir])
-    d.ambient = float(ambient)
+    # the C ABI under test carries these four as float32, so the definition is evaluated (in
+    # double) from the float32-rounded values
+    d.hfov = float(np.float32(hfov))
+    d.light_dir = (C.c_double * 3)(*[float(np.float32(x)) for x in light_dir])
+    d.ambient = float(np.float32(ambient))
     d.sky_rgb = (C.c_uint8 * 3)(*[int(x) for x in sky_rgb])
     d.miss_depth = float(miss_depth)
     return d

@@ -1,0 +1,172 @@
+"""Thin ctypes binding over the C ABI in include/mv.h: argument marshalling only.
+
+torch is used for device memory and streams; every step of the render path runs in the CUDA
+library.  There is no fallback: if `libmv_b200.so` is missing or fails to load, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "libmv_b200.so"
+_lib = None
+
+MV_OK = 0
+FLAG_MATERIAL_CLAMPED, FLAG_BOX_COUNT_CLAMPED, FLAG_BAD_CAMERA, FLAG_DEVICE_TIMEOUT = 1, 2, 4, 8
+EXPORTS = ["mv_create_batch", "mv_upload_worlds", "mv_set_cameras", "mv_render_batch", "mv_step_host",
+           "mv_query_status", "mv_launch_count", "mv_destroy", "mv_status_string"]
+
+
+class BatchDesc(C.Structure):
+    _fields_ = [("num_envs", C.c_int32), ("agents_per_env", C.c_int32),
+                ("grid_x", C.c_int32), ("grid_y", C.c_int32), ("grid_z", C.c_int32),
+                ("max_boxes", C.c_int32), ("width", C.c_int32), ("height", C.c_int32),
+                ("palette_size", C.c_int32), ("hfov_rad", C.c_float), ("light_dir", C.c_float * 3),
+                ("ambient", C.c_float), ("sky_rgb", C.c_uint8 * 3), ("pad", C.c_uint8),
+                ("miss_depth", C.c_float), ("device", C.c_int32)]
+
+
+class MvError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+def lib() -> C.CDLL:
+    """Load the CUDA library (fails loudly when it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise RuntimeError(f"{_LIB_PATH} is missing: run `python -m paper_2107_08170_b200.build` "
+                               "(there is no CPU fallback)")
+        L = C.CDLL(str(_LIB_PATH))
+        vp, i = C.c_void_p, C.c_int
+        L.mv_create_batch.argtypes = [C.POINTER(BatchDesc), C.POINTER(vp)]
+        L.mv_upload_worlds.argtypes = [vp, i, i, vp, vp, vp, vp, vp]
+        L.mv_set_cameras.argtypes = [vp, vp, vp]
+        L.mv_render_batch.argtypes = [vp, vp, vp, vp]
+        L.mv_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        L.mv_query_status.argtypes = [vp, i, vp]
+        L.mv_launch_count.argtypes = [vp]
+        L.mv_launch_count.restype = C.c_int64
+        L.mv_destroy.argtypes = [vp]
+        L.mv_status_string.argtypes = [i]
+        L.mv_status_string.restype = C.c_char_p
+        for n in EXPORTS[:6] + ["mv_destroy"]:
+            getattr(L, n).restype = i
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().mv_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != MV_OK:
+        raise MvError(code, where)
+
+
+def make_desc(num_envs, agents_per_env, grid, max_boxes, width, height, palette_size, hfov_rad=None,
+              light_dir=(0.36, 0.80, 0.48), ambient=0.3, sky_rgb=(127, 178, 229), miss_depth=0.0,
+              device=0) -> BatchDesc:
+    import math
+    d = BatchDesc()
+    d.num_envs, d.agents_per_env = num_envs, agents_per_env
+    d.grid_x, d.grid_y, d.grid_z = grid
+    d.max_boxes, d.width, d.height, d.palette_size = max_boxes, width, height, palette_size
+    d.hfov_rad = math.pi / 2 if hfov_rad is None else hfov_rad
+    d.light_dir = (C.c_float * 3)(*light_dir)
+    d.ambient = ambient
+    d.sky_rgb = (C.c_uint8 * 3)(*sky_rgb)
+    d.miss_depth = miss_depth
+    d.device = device
+    return d
+
+
+def desc_from_config(cfg, device=0) -> BatchDesc:
+    return make_desc(cfg.num_envs, cfg.agents, cfg.grid, cfg.max_boxes, cfg.width, cfg.height,
+                     cfg.palette_size, cfg.hfov_rad, cfg.light_dir, cfg.ambient, cfg.sky_rgb,
+                     cfg.miss_depth, device)
+
+
+def _dptr(t, dtype=None):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    return C.c_void_p(t.data_ptr())
+
+
+def _hptr(t, dtype=None):
+    if t is None:
+        return None
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CPU tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+class Batch:
+    """Handle to one mv_batch.  Methods mirror the C entry points one to one."""
+
+    def __init__(self, desc: BatchDesc):
+        self.desc = desc
+        self._h = C.c_void_p()
+        _check(lib().mv_create_batch(C.byref(desc), C.byref(self._h)), "mv_create_batch")
+        self.num_obs = desc.num_envs * desc.agents_per_env
+
+    def upload_worlds(self, env_begin, env_count, grid=None, boxes=None, box_count=None, palette=None,
+                      stream=None):
+        _check(lib().mv_upload_worlds(self._h, env_begin, env_count, _dptr(grid, torch.uint8),
+                                      _dptr(boxes, torch.int32), _dptr(box_count, torch.int32),
+                                      _dptr(palette, torch.uint8), _stream(stream)), "mv_upload_worlds")
+
+    def set_cameras(self, cams, stream=None):
+        _check(lib().mv_set_cameras(self._h, _dptr(cams, torch.int32), _stream(stream)), "mv_set_cameras")
+
+    def render_batch(self, rgb, depth, stream=None):
+        _check(lib().mv_render_batch(self._h, _dptr(rgb, torch.uint8), _dptr(depth, torch.float32),
+                                     _stream(stream)), "mv_render_batch")
+
+    def step_host(self, cams, rgb, depth, boxes=None, box_count=None, stream=None):
+        _check(lib().mv_step_host(self._h, _hptr(cams, torch.int32), _hptr(boxes, torch.int32),
+                                  _hptr(box_count, torch.int32), _hptr(rgb, torch.uint8),
+                                  _hptr(depth, torch.float32), _stream(stream)), "mv_step_host")
+
+    def query_status(self, clear=False, stream=None) -> int:
+        r = lib().mv_query_status(self._h, int(clear), _stream(stream))
+        if r < 0:
+            raise MvError(r, "mv_query_status")
+        return r
+
+    def launch_count(self) -> int:
+        return int(lib().mv_launch_count(self._h))
+
+    def alloc_outputs(self):
+        dev = torch.device("cuda", self.desc.device)
+        rgb = torch.empty(self.num_obs, self.desc.height, self.desc.width, 3, dtype=torch.uint8, device=dev)
+        depth = torch.empty(self.num_obs, self.desc.height, self.desc.width, dtype=torch.float32, device=dev)
+        return rgb, depth
+
+    def destroy(self):
+        if self._h:
+            h, self._h = self._h, C.c_void_p()
+            _check(lib().mv_destroy(h), "mv_destroy")
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

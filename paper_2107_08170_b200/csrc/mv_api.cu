@@ -1,0 +1,362 @@
+// Host side of the C ABI declared in include/mv.h: argument checks, allocation of the
+// device-resident world store, and the kernel launches.  No rendering arithmetic runs here.
+#include "../../include/mv.h"
+#include "mv_device.cuh"
+#include "mv_pack.cuh"
+#include "mv_render.cuh"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace mv;
+
+namespace {
+
+constexpr int kRenderThreads = 256;
+constexpr int kHostChunks = 8;
+
+inline uint32_t round_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+struct mv_batch {
+    mv_batch_desc desc;
+    int num_obs = 0;
+    size_t nvox = 0;
+    EnvLayout lay{};
+    unsigned char *d_env_blocks = nullptr;
+    uint8_t *d_mat = nullptr;
+    CamRec *d_cams = nullptr;
+    uint32_t *d_status = nullptr;
+    // host-side readiness tracking (per env)
+    std::vector<uint8_t> has_grid, has_palette;
+    int missing_grid = 0, missing_palette = 0;
+    bool has_cams = false;
+    double kr = 0, ku = 0;
+    uint32_t sky_rgbx = 0;
+    uint32_t smem_mask_off = 0, smem_rel_off = 0, smem_misc_off = 0, smem_bytes = 0;
+    int tiles_x = 0, tiles_y = 0, mask_words = 0;
+    int64_t launches = 0;
+    int last_cuda_error = 0;
+    // mv_step_host resources (allocated on first use)
+    uint8_t *d_rgb = nullptr;
+    float *d_depth = nullptr;
+    mv_camera *d_cam_in = nullptr;
+    mv_box *d_box_in = nullptr;
+    int32_t *d_count_in = nullptr;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_chunk[kHostChunks] = {};
+    cudaEvent_t ev_done = nullptr;
+};
+
+namespace {
+
+int cuda_fail(mv_batch *b, cudaError_t e) {
+    if (b) b->last_cuda_error = (int)e;
+    return e == cudaErrorMemoryAllocation ? MV_ERR_OUT_OF_MEMORY : MV_ERR_CUDA;
+}
+
+#define MV_CUDA(b, call)                                   \
+    do {                                                   \
+        cudaError_t e_ = (call);                           \
+        if (e_ != cudaSuccess) return cuda_fail((b), e_);  \
+    } while (0)
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() { if (ok && prev >= 0) cudaSetDevice(prev); }
+};
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int launch_render(mv_batch *b, uint8_t *d_rgb, float *d_depth, int obs_begin, int obs_count, cudaStream_t s) {
+    RenderParams p{};
+    p.env_blocks = b->d_env_blocks;
+    p.mat = b->d_mat;
+    p.cams = b->d_cams;
+    p.rgb = d_rgb;
+    p.depth = d_depth;
+    p.status = b->d_status;
+    p.lay = b->lay;
+    p.obs_begin = obs_begin;
+    p.obs_count = obs_count;
+    p.agents = b->desc.agents_per_env;
+    p.gx = b->desc.grid_x; p.gy = b->desc.grid_y; p.gz = b->desc.grid_z;
+    p.max_boxes = b->desc.max_boxes;
+    p.palette = b->desc.palette_size;
+    p.W = b->desc.width; p.H = b->desc.height;
+    p.tiles_x = b->tiles_x; p.tiles_y = b->tiles_y; p.mask_words = b->mask_words;
+    p.sky_rgbx = b->sky_rgbx;
+    p.miss_depth = b->desc.miss_depth;
+    p.smem_mask_off = b->smem_mask_off; p.smem_rel_off = b->smem_rel_off; p.smem_misc_off = b->smem_misc_off;
+    render_kernel<kRenderThreads><<<obs_count, kRenderThreads, b->smem_bytes, s>>>(p);
+    b->launches++;
+    MV_CUDA(b, cudaGetLastError());
+    return MV_OK;
+}
+
+int launch_cameras(mv_batch *b, const mv_camera *d_cams, cudaStream_t s) {
+    const int n = b->num_obs;
+    camera_kernel<<<(n + 127) / 128, 128, 0, s>>>(reinterpret_cast<const int32_t *>(d_cams), b->d_cams, n,
+                                                   b->kr, b->ku, b->d_status);
+    b->launches++;
+    MV_CUDA(b, cudaGetLastError());
+    b->has_cams = true;
+    return MV_OK;
+}
+
+int launch_boxes(mv_batch *b, int env_begin, int env_count, const mv_box *d_boxes, const int32_t *d_count,
+                 cudaStream_t s) {
+    const int n = env_count * (b->desc.max_boxes + 1);
+    copy_boxes_kernel<<<(n + 255) / 256, 256, 0, s>>>(reinterpret_cast<const uint4 *>(d_boxes), d_count,
+                                                       b->d_env_blocks, b->lay, env_begin, env_count,
+                                                       b->desc.max_boxes, b->desc.palette_size, b->d_status);
+    b->launches++;
+    MV_CUDA(b, cudaGetLastError());
+    return MV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *mv_status_string(int status) {
+    switch (status) {
+        case MV_OK: return "ok";
+        case MV_ERR_INVALID_ARG: return "invalid argument";
+        case MV_ERR_OUT_OF_MEMORY: return "out of memory";
+        case MV_ERR_CUDA: return "CUDA runtime error";
+        case MV_ERR_NOT_READY: return "worlds or cameras not uploaded yet";
+        case MV_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case MV_ERR_UNSUPPORTED: return "configuration exceeds a documented limit";
+        default: return status > 0 ? "data-error flags set" : "unknown status";
+    }
+}
+
+int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
+    if (!desc || !out) return MV_ERR_INVALID_ARG;
+    *out = nullptr;
+    const mv_batch_desc &d = *desc;
+    auto dim_ok = [](int g) { return g >= 4 && g <= 1024 && (g % 4) == 0; };
+    if (d.num_envs < 1 || d.agents_per_env < 1 || !dim_ok(d.grid_x) || !dim_ok(d.grid_y) || !dim_ok(d.grid_z) ||
+        d.max_boxes < 0 || d.max_boxes > 256 || d.width < 8 || d.width > 4096 || (d.width % 8) != 0 ||
+        d.height < 4 || d.height > 4096 || (d.height % 4) != 0 || d.palette_size < 1 || d.palette_size > 256 ||
+        !(d.hfov_rad > 0.0f) || !(d.hfov_rad < 3.14159f) || !(d.ambient >= 0.0f) || !(d.ambient <= 1.0f) ||
+        !std::isfinite(d.miss_depth) || d.device < 0)
+        return MV_ERR_INVALID_ARG;
+    const double ln = (double)d.light_dir[0] * d.light_dir[0] + (double)d.light_dir[1] * d.light_dir[1] +
+                      (double)d.light_dir[2] * d.light_dir[2];
+    if (!(ln > 0.0) || !std::isfinite(ln)) return MV_ERR_INVALID_ARG;
+    if ((int64_t)d.num_envs * d.agents_per_env > (1 << 30)) return MV_ERR_INVALID_ARG;
+
+    mv_batch *b = new (std::nothrow) mv_batch();
+    if (!b) return MV_ERR_OUT_OF_MEMORY;
+    b->desc = d;
+    b->num_obs = d.num_envs * d.agents_per_env;
+    b->nvox = (size_t)d.grid_x * d.grid_y * d.grid_z;
+    b->has_grid.assign(d.num_envs, 0);
+    b->has_palette.assign(d.num_envs, 0);
+    b->missing_grid = b->missing_palette = d.num_envs;
+
+    EnvLayout &L = b->lay;
+    L.occ_bytes = round_up((uint32_t)(b->nvox / 8), 16);
+    L.lut_off = L.occ_bytes;
+    L.box_off = L.lut_off + round_up(kFaces * d.palette_size * 4, 16);
+    L.count_off = L.box_off + (uint32_t)d.max_boxes * 32;
+    L.block_bytes = L.count_off + 16;
+    L.stride = round_up(L.block_bytes, 128);
+
+    b->tiles_x = d.width / 8;
+    b->tiles_y = d.height / 4;
+    b->mask_words = d.max_boxes > 0 ? (d.max_boxes + 31) / 32 : 1;
+    b->smem_mask_off = round_up(L.block_bytes, 16);
+    b->smem_rel_off = b->smem_mask_off + round_up((uint32_t)(b->tiles_x * b->tiles_y * b->mask_words * 4), 16);
+    b->smem_misc_off = b->smem_rel_off + (uint32_t)(d.max_boxes > 0 ? d.max_boxes : 1) * 32;
+    b->smem_bytes = b->smem_misc_off + 16;
+
+    // kr = tan(hfov/2)/W, ku = (tan(hfov/2)*H/W)/H in double (scalar set-up for the camera kernel)
+    const double tx = std::tan((double)d.hfov_rad / 2.0);
+    const double ty = tx * (double)d.height / (double)d.width;
+    b->kr = tx / (double)d.width;
+    b->ku = ty / (double)d.height;
+    b->sky_rgbx = (uint32_t)d.sky_rgb[0] | ((uint32_t)d.sky_rgb[1] << 8) | ((uint32_t)d.sky_rgb[2] << 16);
+
+    int ndev = 0;
+    cudaError_t e = cudaGetDeviceCount(&ndev);
+    if (e != cudaSuccess || d.device >= ndev) { delete b; return e != cudaSuccess ? MV_ERR_CUDA : MV_ERR_INVALID_ARG; }
+    DeviceGuard g(d.device);
+    if (!g.ok) { delete b; return MV_ERR_CUDA; }
+    int smem_max = 0;
+    e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, d.device);
+    if (e != cudaSuccess) { delete b; return MV_ERR_CUDA; }
+    if ((int)b->smem_bytes > smem_max) { delete b; return MV_ERR_UNSUPPORTED; }
+    e = cudaFuncSetAttribute(render_kernel<kRenderThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)b->smem_bytes);
+    if (e != cudaSuccess) { delete b; return MV_ERR_CUDA; }
+
+    const size_t blocks_bytes = (size_t)d.num_envs * L.stride;
+    bool ok = cudaMalloc(&b->d_env_blocks, blocks_bytes) == cudaSuccess &&
+              cudaMalloc(&b->d_mat, (size_t)d.num_envs * b->nvox) == cudaSuccess &&
+              cudaMalloc(&b->d_cams, (size_t)b->num_obs * sizeof(CamRec)) == cudaSuccess &&
+              cudaMalloc(&b->d_status, 16) == cudaSuccess;
+    if (ok) ok = cudaMemset(b->d_env_blocks, 0, blocks_bytes) == cudaSuccess &&
+                 cudaMemset(b->d_status, 0, 16) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        mv_destroy(b);
+        return MV_ERR_OUT_OF_MEMORY;
+    }
+    *out = b;
+    return MV_OK;
+}
+
+int mv_upload_worlds(mv_batch *b, int env_begin, int env_count, const uint8_t *d_grid, const mv_box *d_boxes,
+                     const int32_t *d_box_count, const uint8_t *d_palette, void *cuda_stream) {
+    if (!b || env_begin < 0 || env_count < 0 || (int64_t)env_begin + env_count > b->desc.num_envs)
+        return MV_ERR_INVALID_ARG;
+    if (d_boxes && !d_box_count) return MV_ERR_INVALID_ARG;
+    if (d_boxes && b->desc.max_boxes == 0) return MV_ERR_INVALID_ARG;
+    if ((d_grid && !aligned16(d_grid)) || (d_boxes && !aligned16(d_boxes))) return MV_ERR_INVALID_ARG;
+    if (env_count == 0) return MV_OK;
+    DeviceGuard g(b->desc.device);
+    if (!g.ok) return MV_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (d_grid) {
+        const size_t threads = b->nvox / 32 * (size_t)env_count;
+        const size_t blocks = (threads + 255) / 256;
+        if (blocks > 0x7fffffffull) return MV_ERR_INVALID_ARG;
+        pack_grid_kernel<<<(unsigned)blocks, 256, 0, s>>>(d_grid, b->d_env_blocks, b->d_mat, b->lay, b->nvox,
+                                                           env_begin, env_count, b->desc.palette_size, b->d_status);
+        b->launches++;
+        MV_CUDA(b, cudaGetLastError());
+        for (int e = env_begin; e < env_begin + env_count; ++e)
+            if (!b->has_grid[e]) { b->has_grid[e] = 1; b->missing_grid--; }
+    }
+    if (d_palette) {
+        const int n = env_count * kFaces * b->desc.palette_size;
+        build_lut_kernel<<<(n + 255) / 256, 256, 0, s>>>(d_palette, b->d_env_blocks, b->lay, env_begin, env_count,
+                                                          b->desc.palette_size, (double)b->desc.light_dir[0],
+                                                          (double)b->desc.light_dir[1], (double)b->desc.light_dir[2],
+                                                          (double)b->desc.ambient);
+        b->launches++;
+        MV_CUDA(b, cudaGetLastError());
+        for (int e = env_begin; e < env_begin + env_count; ++e)
+            if (!b->has_palette[e]) { b->has_palette[e] = 1; b->missing_palette--; }
+    }
+    if (d_boxes) {
+        int r = launch_boxes(b, env_begin, env_count, d_boxes, d_box_count, s);
+        if (r != MV_OK) return r;
+    }
+    return MV_OK;
+}
+
+int mv_set_cameras(mv_batch *b, const mv_camera *d_cams, void *cuda_stream) {
+    if (!b || !d_cams) return MV_ERR_INVALID_ARG;
+    DeviceGuard g(b->desc.device);
+    if (!g.ok) return MV_ERR_CUDA;
+    return launch_cameras(b, d_cams, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int mv_render_batch(mv_batch *b, uint8_t *d_rgb, float *d_depth, void *cuda_stream) {
+    if (!b || !d_rgb || !d_depth || !aligned16(d_rgb) || !aligned16(d_depth)) return MV_ERR_INVALID_ARG;
+    if (b->missing_grid > 0 || b->missing_palette > 0 || !b->has_cams) return MV_ERR_NOT_READY;
+    DeviceGuard g(b->desc.device);
+    if (!g.ok) return MV_ERR_CUDA;
+    return launch_render(b, d_rgb, d_depth, 0, b->num_obs, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int mv_step_host(mv_batch *b, const mv_camera *h_cams, const mv_box *h_boxes, const int32_t *h_box_count,
+                 uint8_t *h_rgb, float *h_depth, void *cuda_stream) {
+    if (!b || !h_cams || !h_rgb || !h_depth) return MV_ERR_INVALID_ARG;
+    if (h_boxes && (!h_box_count || b->desc.max_boxes == 0)) return MV_ERR_INVALID_ARG;
+    if (b->missing_grid > 0 || b->missing_palette > 0) return MV_ERR_NOT_READY;
+    DeviceGuard g(b->desc.device);
+    if (!g.ok) return MV_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t px = (size_t)b->desc.width * b->desc.height;
+    const int E = b->desc.num_envs, O = b->num_obs;
+    if (!b->d_rgb) {
+        MV_CUDA(b, cudaMalloc(&b->d_rgb, (size_t)O * px * 3));
+        MV_CUDA(b, cudaMalloc(&b->d_depth, (size_t)O * px * 4));
+        MV_CUDA(b, cudaMalloc(&b->d_cam_in, (size_t)O * sizeof(mv_camera)));
+        if (b->desc.max_boxes > 0) {
+            MV_CUDA(b, cudaMalloc(&b->d_box_in, (size_t)E * b->desc.max_boxes * sizeof(mv_box)));
+            MV_CUDA(b, cudaMalloc(&b->d_count_in, (size_t)E * sizeof(int32_t)));
+        }
+        MV_CUDA(b, cudaStreamCreateWithFlags(&b->copy_stream, cudaStreamNonBlocking));
+        for (auto &ev : b->ev_chunk) MV_CUDA(b, cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+        MV_CUDA(b, cudaEventCreateWithFlags(&b->ev_done, cudaEventDisableTiming));
+    }
+    MV_CUDA(b, cudaMemcpyAsync(b->d_cam_in, h_cams, (size_t)O * sizeof(mv_camera), cudaMemcpyHostToDevice, s));
+    if (h_boxes) {
+        MV_CUDA(b, cudaMemcpyAsync(b->d_box_in, h_boxes, (size_t)E * b->desc.max_boxes * sizeof(mv_box),
+                                   cudaMemcpyHostToDevice, s));
+        MV_CUDA(b, cudaMemcpyAsync(b->d_count_in, h_box_count, (size_t)E * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+        int r = launch_boxes(b, 0, E, b->d_box_in, b->d_count_in, s);
+        if (r != MV_OK) return r;
+    }
+    int r = launch_cameras(b, b->d_cam_in, s);
+    if (r != MV_OK) return r;
+    // render chunk by chunk; each chunk's frames start their trip to the host while the next renders
+    const int chunks = O < kHostChunks ? 1 : kHostChunks;
+    for (int c = 0; c < chunks; ++c) {
+        const int o0 = (int)((int64_t)O * c / chunks), o1 = (int)((int64_t)O * (c + 1) / chunks);
+        r = launch_render(b, b->d_rgb, b->d_depth, o0, o1 - o0, s);
+        if (r != MV_OK) return r;
+        MV_CUDA(b, cudaEventRecord(b->ev_chunk[c], s));
+        MV_CUDA(b, cudaStreamWaitEvent(b->copy_stream, b->ev_chunk[c], 0));
+        MV_CUDA(b, cudaMemcpyAsync(h_rgb + (size_t)o0 * px * 3, b->d_rgb + (size_t)o0 * px * 3,
+                                   (size_t)(o1 - o0) * px * 3, cudaMemcpyDeviceToHost, b->copy_stream));
+        MV_CUDA(b, cudaMemcpyAsync(h_depth + (size_t)o0 * px, b->d_depth + (size_t)o0 * px,
+                                   (size_t)(o1 - o0) * px * 4, cudaMemcpyDeviceToHost, b->copy_stream));
+    }
+    MV_CUDA(b, cudaEventRecord(b->ev_done, b->copy_stream));
+    MV_CUDA(b, cudaStreamWaitEvent(s, b->ev_done, 0));
+    MV_CUDA(b, cudaStreamSynchronize(s));
+    return MV_OK;
+}
+
+int mv_query_status(mv_batch *b, int clear, void *cuda_stream) {
+    if (!b) return MV_ERR_INVALID_ARG;
+    DeviceGuard g(b->desc.device);
+    if (!g.ok) return MV_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    uint32_t word = 0;
+    MV_CUDA(b, cudaMemcpyAsync(&word, b->d_status, 4, cudaMemcpyDeviceToHost, s));
+    if (clear) MV_CUDA(b, cudaMemsetAsync(b->d_status, 0, 4, s));
+    MV_CUDA(b, cudaStreamSynchronize(s));
+    if (word & kFlagTimeout) return MV_ERR_DEVICE_TIMEOUT;
+    return (int)word;
+}
+
+int64_t mv_launch_count(const mv_batch *b) { return b ? b->launches : 0; }
+
+int mv_destroy(mv_batch *b) {
+    if (!b) return MV_OK;
+    int rc = MV_OK;
+    {
+        DeviceGuard g(b->desc.device);
+        if (g.ok) {
+            if (cudaDeviceSynchronize() != cudaSuccess) rc = MV_ERR_CUDA;
+            cudaFree(b->d_env_blocks); cudaFree(b->d_mat); cudaFree(b->d_cams); cudaFree(b->d_status);
+            cudaFree(b->d_rgb); cudaFree(b->d_depth); cudaFree(b->d_cam_in); cudaFree(b->d_box_in);
+            cudaFree(b->d_count_in);
+            if (b->copy_stream) cudaStreamDestroy(b->copy_stream);
+            for (auto &ev : b->ev_chunk) if (ev) cudaEventDestroy(ev);
+            if (b->ev_done) cudaEventDestroy(b->ev_done);
+            cudaGetLastError();
+        }
+    }
+    delete b;
+    return rc;
+}
+
+}  // extern "C"

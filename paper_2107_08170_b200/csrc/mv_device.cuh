@@ -1,0 +1,55 @@
+// Device-side data layout shared by the pack, camera and render kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mv {
+
+// Face codes: 0..5 = -x,+x,-y,+y,-z,+z (outward normal), 6 = camera inside the solid.
+constexpr int kFaces = 7;
+constexpr int kFaceInside = 6;
+
+constexpr uint32_t kFlagMaterial = 0x1u;
+constexpr uint32_t kFlagBoxCount = 0x2u;
+constexpr uint32_t kFlagBadCamera = 0x4u;
+constexpr uint32_t kFlagTimeout = 0x8u;
+
+// Per-observation ray basis written by the camera kernel (64 bytes, one 128-bit lane each).
+struct __align__(16) CamRec {
+    float P[3], F[3], Rs[3], Us[3];   // eye, unit forward, per-half-pixel right and up steps
+    int32_t self_box;
+    uint32_t flags;                   // kFlagBadCamera when a component was not finite
+    uint32_t pad[2];
+};
+static_assert(sizeof(CamRec) == 64, "CamRec must be 64 bytes");
+
+// One environment's render inputs, contiguous in HBM so that a single bulk copy stages them
+// into shared memory:  [occupancy bits | shade LUT | boxes | box count].
+struct EnvLayout {
+    uint32_t occ_bytes;     // grid_x*grid_y*grid_z/8 rounded up to 16
+    uint32_t lut_off;       // 7*palette_size RGBX words
+    uint32_t box_off;       // max_boxes * 32 bytes
+    uint32_t count_off;     // 16 bytes, first int32 = box count
+    uint32_t block_bytes;   // bytes staged per CTA (multiple of 16)
+    uint32_t stride;        // distance between envs in HBM (multiple of 128)
+};
+
+struct RenderParams {
+    const unsigned char *env_blocks;   // [E] EnvLayout blocks
+    const uint8_t *mat;                // [E][nvox] material ids (clamped to palette at upload)
+    const CamRec *cams;                // [O]
+    uint8_t *rgb;                      // [O][H][W][3]
+    float *depth;                      // [O][H][W]
+    uint32_t *status;
+    EnvLayout lay;
+    int obs_begin, obs_count;
+    int agents;
+    int gx, gy, gz;
+    int max_boxes, palette;
+    int W, H, tiles_x, tiles_y, mask_words;
+    uint32_t sky_rgbx;
+    float miss_depth;
+    uint32_t smem_mask_off, smem_rel_off, smem_misc_off;   // offsets after the env block
+};
+
+}  // namespace mv

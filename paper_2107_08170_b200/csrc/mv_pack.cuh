@@ -1,0 +1,128 @@
+// World-store and camera kernels: everything that turns the caller's arrays into the
+// device-resident layout the render kernel stages (paper Section 3.3: geometry is prepared
+// once per episode; Section 3.2: objects and cameras are state that changes every step).
+#pragma once
+#include "mv_device.cuh"
+
+namespace mv {
+
+// Four 0/non-zero bytes of a word -> 4 bits.
+__device__ __forceinline__ uint32_t nz_bits4(uint32_t v) {
+    const uint32_t ones = __vcmpne4(v, 0u) & 0x01010101u;
+    return (ones * 0x01020408u) >> 24;
+}
+
+// uint8 grid [env][y][z][x] -> 1 bit per voxel (bit v&31 of word v>>5, v = x + gx*(z + gz*y))
+// inside the env block, plus a material copy with ids clamped to the palette.  One thread
+// packs 32 voxels.
+__global__ void pack_grid_kernel(const uint8_t *__restrict__ grid, unsigned char *__restrict__ env_blocks,
+                                 uint8_t *__restrict__ mat, EnvLayout lay, size_t nvox, int env_begin,
+                                 int env_count, int palette, uint32_t *status)
+{
+    const size_t words_per_env = nvox / 32;
+    const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (gid >= words_per_env * (size_t)env_count) return;
+    const size_t e = gid / words_per_env, w = gid - e * words_per_env;
+    const uint4 *src = reinterpret_cast<const uint4 *>(grid + e * nvox + w * 32);
+    uint4 q[2] = {src[0], src[1]};
+    uint32_t *v = reinterpret_cast<uint32_t *>(q);
+    const uint32_t cap = (uint32_t)(palette - 1) * 0x01010101u;
+    uint32_t bits = 0, clamped = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t orig = v[i];
+        bits |= nz_bits4(orig) << (4 * i);          // filled = id != 0, decided before clamping
+        const uint32_t c = __vminu4(orig, cap);
+        clamped |= c ^ orig;
+        v[i] = c;
+    }
+    const size_t env = (size_t)env_begin + e;
+    reinterpret_cast<uint32_t *>(env_blocks + env * lay.stride)[w] = bits;
+    uint4 *dst = reinterpret_cast<uint4 *>(mat + env * nvox + w * 32);
+    dst[0] = q[0];
+    dst[1] = q[1];
+    if (clamped) atomicOr(status, kFlagMaterial);
+}
+
+// Shaded colour table per env: lut[face][m] = RGBX of floor(palette*I_face + 0.5), in double.
+__global__ void build_lut_kernel(const uint8_t *__restrict__ palette, unsigned char *__restrict__ env_blocks,
+                                 EnvLayout lay, int env_begin, int env_count, int P,
+                                 double lx, double ly, double lz, double ambient)
+{
+    const int gid = blockIdx.x * blockDim.x + threadIdx.x;
+    if (gid >= env_count * kFaces * P) return;
+    const int e = gid / (kFaces * P), r = gid - e * kFaces * P;
+    const int f = r / P, m = r - f * P;
+    double I = ambient;
+    if (f < 6) {
+        const double n = sqrt(__dadd_rn(__dadd_rn(__dmul_rn(lx, lx), __dmul_rn(ly, ly)), __dmul_rn(lz, lz)));
+        const double comp = (f >> 1) == 0 ? lx : ((f >> 1) == 1 ? ly : lz);
+        double l = comp / n;
+        if (!(f & 1)) l = -l;                       // even faces have the negative normal
+        l = l > 0.0 ? l : 0.0;
+        I = __dadd_rn(ambient, __dmul_rn(__dsub_rn(1.0, ambient), l));
+    }
+    const uint8_t *pc = palette + ((size_t)e * P + m) * 3;
+    uint32_t out = 0;
+#pragma unroll
+    for (int c = 0; c < 3; ++c) {
+        double v = floor(__dadd_rn(__dmul_rn((double)pc[c], I), 0.5));
+        v = v > 255.0 ? 255.0 : v;
+        out |= (uint32_t)v << (8 * c);
+    }
+    uint32_t *lut = reinterpret_cast<uint32_t *>(env_blocks + (size_t)(env_begin + e) * lay.stride + lay.lut_off);
+    lut[f * P + m] = out;
+}
+
+// Box lists into the env blocks; material ids and counts are clamped.
+__global__ void copy_boxes_kernel(const uint4 *__restrict__ boxes, const int32_t *__restrict__ counts,
+                                  unsigned char *__restrict__ env_blocks, EnvLayout lay, int env_begin,
+                                  int env_count, int max_boxes, int palette, uint32_t *status)
+{
+    const int gid = blockIdx.x * blockDim.x + threadIdx.x;
+    const int per_env = max_boxes + 1;
+    if (gid >= env_count * per_env) return;
+    const int e = gid / per_env, b = gid - e * per_env;
+    unsigned char *blk = env_blocks + (size_t)(env_begin + e) * lay.stride;
+    if (b == max_boxes) {
+        int n = counts[e];
+        if (n < 0 || n > max_boxes) { n = n < 0 ? 0 : max_boxes; atomicOr(status, kFlagBoxCount); }
+        *reinterpret_cast<int4 *>(blk + lay.count_off) = make_int4(n, 0, 0, 0);
+        return;
+    }
+    uint4 lo = boxes[((size_t)e * max_boxes + b) * 2], hi = boxes[((size_t)e * max_boxes + b) * 2 + 1];
+    if (hi.z >= (uint32_t)palette) { hi.z = palette - 1; atomicOr(status, kFlagMaterial); }
+    uint4 *dst = reinterpret_cast<uint4 *>(blk + lay.box_off) + 2 * b;
+    dst[0] = lo;
+    dst[1] = hi;
+}
+
+// Camera -> ray basis, evaluated in double and rounded to float:
+// F = (cp*sy, sp, cp*cy), R = (cy, 0, -sy), U = (-sp*sy, cp, -sp*cy); Rs = R*kr, Us = U*ku
+// with kr = tan(hfov/2)/W and ku = (tan(hfov/2)*H/W)/H computed on the host in double.
+__global__ void camera_kernel(const int32_t *__restrict__ cams, CamRec *__restrict__ out, int num_obs,
+                              double kr, double ku, uint32_t *status)
+{
+    const int o = blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= num_obs) return;
+    const int32_t *c = cams + (size_t)o * 6;
+    const float px = __int_as_float(c[0]), py = __int_as_float(c[1]), pz = __int_as_float(c[2]);
+    const float yaw = __int_as_float(c[3]), pitch = __int_as_float(c[4]);
+    CamRec r;
+    r.self_box = c[5];
+    r.pad[0] = r.pad[1] = 0;
+    const bool ok = isfinite(px) && isfinite(py) && isfinite(pz) && isfinite(yaw) && isfinite(pitch);
+    r.flags = ok ? 0u : kFlagBadCamera;
+    double sy, cy, sp, cp;
+    sincos((double)(ok ? yaw : 0.0f), &sy, &cy);
+    sincos((double)(ok ? pitch : 0.0f), &sp, &cp);
+    r.P[0] = px; r.P[1] = py; r.P[2] = pz;
+    r.F[0] = (float)__dmul_rn(cp, sy); r.F[1] = (float)sp; r.F[2] = (float)__dmul_rn(cp, cy);
+    r.Rs[0] = (float)__dmul_rn(cy, kr); r.Rs[1] = (float)__dmul_rn(0.0, kr); r.Rs[2] = (float)__dmul_rn(-sy, kr);
+    r.Us[0] = (float)__dmul_rn(__dmul_rn(-sp, sy), ku); r.Us[1] = (float)__dmul_rn(cp, ku);
+    r.Us[2] = (float)__dmul_rn(__dmul_rn(-sp, cy), ku);
+    out[o] = r;
+    if (!ok) atomicOr(status, kFlagBadCamera);
+}
+
+}  // namespace mv

@@ -1,0 +1,306 @@
+"""CUDA path (through the C ABI) against the CPU oracle, element by element."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from helpers import cam_row, box_rows
+from paper_2107_08170_b200 import scenes
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _binding():
+    from paper_2107_08170_b200 import binding
+    return binding
+
+
+def _render_custom(oracle, grid, palette, cams, W, H, boxes=None, box_count=None, agents=1, max_boxes=0,
+                   check=True, **desc_kw):
+    """One env-batch of hand-made worlds: grid [E][gy][gz][gx], cams [E*agents][6]."""
+    B = _binding()
+    E, gy, gz, gx = grid.shape
+    P = palette.shape[1]
+    desc = B.make_desc(E, agents, (gx, gy, gz), max_boxes, W, H, P, **desc_kw)
+    batch = B.Batch(desc)
+    dev = torch.device("cuda", 0)
+    t = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a)).to(dt).to(dev)
+    bt = ct = None
+    if max_boxes > 0:
+        bt, ct = t(boxes, torch.int32), t(box_count, torch.int32)
+    batch.upload_worlds(0, E, t(grid, torch.uint8), bt, ct, t(palette, torch.uint8))
+    batch.set_cameras(t(cams, torch.int32))
+    rgb, depth = batch.alloc_outputs()
+    batch.render_batch(rgb, depth)
+    status = batch.query_status()
+    g_rgb, g_depth = rgb.cpu().numpy(), depth.cpu().numpy()
+    batch.destroy()
+    if not check:
+        return g_rgb, g_depth, status
+    od = oracle.make_desc((gy, gz, gx), max_boxes, W, H, P, **desc_kw)
+    total = None
+    for o in range(E * agents):
+        e = o // agents
+        bx = boxes[e] if max_boxes > 0 else None
+        bc = int(box_count[e]) if max_boxes > 0 else 0
+        o_rgb, o_depth, o_ids = oracle.render_obs(od, grid[e], bx, bc, palette[e], cams[o])
+        st = parity.compare_obs(oracle, od, grid[e], bx, bc, palette[e], cams[o], g_rgb[o], g_depth[o],
+                                o_rgb, o_depth, o_ids)
+        total = st if total is None else {k: total[k] + st[k] for k in st}
+    return g_rgb, g_depth, status, total
+
+
+def _pal(E, P, seed=0):
+    return np.random.default_rng(seed).integers(20, 255, size=(E, P, 3)).astype(np.uint8)
+
+
+def test_tiny_config_all_pixels(oracle):
+    from gpu_util import render_scene, scene_to_numpy
+    cfg = scenes.config("tiny")
+    sc = scenes.make_scene(cfg)
+    g_rgb, g_depth, status = render_scene(cfg, sc)
+    assert status == 0
+    st = parity.compare_scene(oracle, cfg, scene_to_numpy(sc), range(cfg.num_obs), g_rgb, g_depth)
+    parity.assert_parity(st, "tiny")
+    assert st["pixels"] == 4 * 64 * 36
+
+
+def test_tiny_many_seeds_brute_force(oracle):
+    from gpu_util import render_scene, scene_to_numpy
+    tot = {"pixels": 0, "rgb_mismatch": 0, "unexcused": 0}
+    for seed in range(10, 16):
+        cfg = scenes.config("tiny", seed=seed, num_envs=6)
+        sc = scenes.make_scene(cfg)
+        g_rgb, g_depth, status = render_scene(cfg, sc)
+        st = parity.compare_scene(oracle, cfg, scene_to_numpy(sc), range(cfg.num_obs), g_rgb, g_depth)
+        assert st["unexcused"] == 0, (seed, st)
+        for k in tot:
+            tot[k] += st[k]
+    parity.assert_parity(tot, "tiny seeds")
+
+
+def test_handmade_wall_floor_and_empty(oracle):
+    gx, gy, gz, W, H = 32, 8, 16, 32, 20
+    grid = np.zeros((3, gy, gz, gx), np.uint8)
+    grid[0, 0] = 1; grid[0, :, 12, :] = 1            # floor + wall
+    grid[2] = 1                                       # env 2 solid: camera inside
+    pal = _pal(3, 4)
+    cams = np.stack([cam_row(16.3, 1.5, 2.6, 0.0, 0.0), cam_row(5.2, 3.1, 4.4, 0.7, 0.2),
+                     cam_row(7.5, 3.5, 8.5, 1.0, -0.2)])
+    g_rgb, g_depth, status, st = _render_custom(oracle, grid, pal, cams, W, H, miss_depth=-1.0)
+    assert status == 0 and st["rgb_mismatch"] == 0 and st["depth_mismatch"] == 0
+    assert np.allclose(g_depth[0, : H // 2], 12 - np.float32(2.6), atol=1e-6)      # planar wall depth
+    assert (g_rgb[1] == np.array([127, 178, 229], np.uint8)).all() and (g_depth[1] == -1.0).all()
+    assert (g_depth[2] == 0.0).all()
+    assert (g_rgb[2] == np.floor(pal[2, 1] * np.float64(np.float32(0.3)) + 0.5).astype(np.uint8)).all()
+
+
+def test_mirror_scene_bit_exact(oracle):
+    rng = np.random.default_rng(7)
+    gx, gy, gz, W, H = 16, 8, 16, 48, 28
+    half = rng.integers(0, 6, size=(gy, gz, gx // 2)).astype(np.uint8)
+    half[half > 3] = 0
+    half[:, :, -1] = 0
+    grid = np.concatenate([half, half[:, :, ::-1]], axis=2)[None].copy()
+    grid[0, 0] = 2
+    pal = _pal(1, 4)
+    boxes = box_rows([((6.5, 1.0, 5.0), (7.25, 1.5, 5.5), 1), ((8.75, 1.0, 5.0), (9.5, 1.5, 5.5), 1)])[None]
+    cams = cam_row(gx / 2, 1.5, 1.5, 0.0, 0.1)[None]
+    g_rgb, g_depth, status, st = _render_custom(oracle, grid, pal, cams, W, H, boxes=boxes,
+                                                box_count=np.array([2]), max_boxes=2, light_dir=(0.0, 0.8, 0.6))
+    assert st["unexcused"] == 0
+    assert (g_rgb[0] == g_rgb[0][:, ::-1]).all() and (g_depth[0] == g_depth[0][:, ::-1]).all()
+
+
+def test_camera_outside_grid_and_far_away(oracle):
+    rng = np.random.default_rng(11)
+    gx, gy, gz, W, H = 16, 8, 12, 64, 36
+    grid = ((rng.random((1, gy, gz, gx)) < 0.2) * rng.integers(1, 4, size=(1, gy, gz, gx))).astype(np.uint8)
+    grid = np.repeat(grid, 6, axis=0)
+    pal = np.repeat(_pal(1, 4), 6, axis=0)
+    look = lambda p, q: (math.atan2(q[0] - p[0], q[2] - p[2]),
+                         math.atan2(q[1] - p[1], math.hypot(q[0] - p[0], q[2] - p[2])))
+    c = (8.0, 4.0, 6.0)
+    eyes = [(-6.3, 5.2, -4.1), (24.7, 3.3, 6.2), (8.2, 19.5, 6.4), (8.1, -7.5, 5.7), (16.0, 4.5, 6.5), (-40.0, 12.0, 30.0)]
+    boxes = np.repeat(box_rows([((-3.0, 2.0, -2.0), (-1.5, 3.0, -1.0), 2), ((17.0, 1.0, 5.0), (19.0, 6.0, 7.5), 3)])[None], 6, 0)
+    cams = np.stack([cam_row(*e, *look(e, c)) for e in eyes])
+    g_rgb, g_depth, status, st = _render_custom(oracle, grid, pal, cams, W, H, boxes=boxes,
+                                                box_count=np.full(6, 2), max_boxes=2)
+    parity.assert_parity(st, "outside")
+    assert (g_depth > 0).mean() > 0.15
+
+
+def test_boxes_selfbox_degenerate_and_many_boxes(oracle):
+    rng = np.random.default_rng(21)
+    gx, gy, gz, W, H = 24, 8, 24, 96, 56
+    E, nb, A = 3, 70, 2
+    grid = np.zeros((E, gy, gz, gx), np.uint8); grid[:, 0] = 1
+    grid[:, 1:4, 20, :] = 2
+    pal = _pal(E, 8)
+    items = []
+    for e in range(E):
+        rows = []
+        for b in range(nb):
+            c = rng.uniform([2, 1, 2], [22, 3, 19]); s = rng.uniform(0.2, 1.2, 3)
+            rows.append((c - s / 2, c + s / 2, int(rng.integers(1, 8))))
+        rows[5] = ((3.0, 1.0, 3.0), (3.0, 2.0, 4.0), 1)            # zero width: ignored
+        rows[6] = ((5.0, 2.0, 3.0), (4.0, 3.0, 4.0), 1)            # inverted: ignored
+        items.append(box_rows(rows))
+    boxes = np.stack(items)
+    count = np.array([nb, nb - 7, 0])
+    cams = []
+    for e in range(E):
+        for a in range(A):
+            x, z = rng.uniform(4, 20), rng.uniform(3, 10)
+            bid = 10 + a
+            body = box_rows([((x - .25, 1.0, z - .25), (x + .25, 2.0, z + .25), 3)])[0]
+            boxes[e, bid] = body
+            cams.append(cam_row(x, 1.75, z, rng.uniform(-0.6, 0.6), rng.uniform(-0.3, 0.2), self_box=bid))
+    cams = np.stack(cams)
+    g_rgb, g_depth, status, st = _render_custom(oracle, grid, pal, cams, W, H, boxes=boxes, box_count=count,
+                                                agents=A, max_boxes=nb)
+    parity.assert_parity(st, "boxes")
+    assert status == 0
+
+
+def test_voxel_as_box_and_axis_parallel_rays(oracle):
+    """Boxes equal to voxel cells render like those voxels; yaw=pitch=0 gives rays with exact zeros
+    in no component but exercises the aligned case; a camera on a voxel boundary plane too."""
+    rng = np.random.default_rng(3)
+    g = 8
+    W, H = 40, 24
+    cells = [(2, 3, 5), (5, 1, 6), (6, 4, 2), (3, 3, 3), (1, 1, 6)]
+    grid = np.zeros((2, g, g, g), np.uint8)
+    rows = []
+    for n, (i, j, k) in enumerate(cells):
+        grid[0, j, k, i] = 1 + n % 3
+        rows.append(((i, j, k), (i + 1, j + 1, k + 1), 1 + n % 3))
+    boxes = np.stack([box_rows(rows), box_rows(rows)])
+    pal = np.repeat(_pal(1, 4), 2, axis=0)
+    cams = np.stack([cam_row(0.7, 2.6, 0.4, 0.75, 0.05)] * 2)
+    g_rgb, g_depth, status, st = _render_custom(oracle, grid, pal, cams, W, H, boxes=boxes,
+                                                box_count=np.array([0, 5]), max_boxes=5)
+    parity.assert_parity(st, "voxel-as-box")
+    same = (g_rgb[0] == g_rgb[1]).all(axis=-1) & parity.depth_close(g_depth[0], g_depth[1])
+    assert same.mean() > 0.995
+    # aligned camera on a boundary plane (x = 4.0), cells next to the plane empty
+    grid2 = np.zeros((1, g, g, g), np.uint8); grid2[0, 0] = 1; grid2[0, :, 7, :] = 2; grid2[0, 1:3, 4, 1] = 3; grid2[0, 1:3, 4, 6] = 3
+    cams2 = cam_row(4.0, 1.5, 0.5, 0.0, 0.0)[None]
+    _, _, _, st2 = _render_custom(oracle, grid2, _pal(1, 4), cams2, W, H)
+    parity.assert_parity(st2, "aligned")
+    assert st2["rgb_mismatch"] == 0
+
+
+def test_data_errors_set_flags_and_stay_in_bounds(oracle):
+    B = _binding()
+    gx, gy, gz, W, H = 8, 8, 8, 16, 8
+    grid = np.zeros((2, gy, gz, gx), np.uint8); grid[:, 0] = 200; grid[:, :, 7, :] = 3
+    pal = _pal(2, 4)
+    boxes = np.stack([box_rows([((2, 1, 4), (3, 2, 5), 77), ((5, 1, 4), (6, 2, 5), 1)])] * 2)
+    count = np.array([9, -3])
+    cams = np.stack([cam_row(4.5, 2.5, 1.5, 0.0, 0.0), cam_row(float("nan"), 2.5, 1.5, 0.0, 0.0)])
+    g_rgb, g_depth, status, st = _render_custom(oracle, grid, pal, cams, W, H, boxes=boxes, box_count=count,
+                                                max_boxes=2)
+    assert status == (B.FLAG_MATERIAL_CLAMPED | B.FLAG_BOX_COUNT_CLAMPED | B.FLAG_BAD_CAMERA)
+    assert st["rgb_mismatch"] == 0 and st["depth_mismatch"] == 0
+    assert (g_rgb[1] == np.array([127, 178, 229], np.uint8)).all()
+
+
+@pytest.mark.parametrize("name,envs", [("rooms", 6), ("rooms_boxes", 3), ("headline", 5), ("sweep", 3)])
+def test_workload_shapes_small_batches(oracle, name, envs):
+    from gpu_util import render_scene, scene_to_numpy
+    cfg = scenes.config(name, num_envs=envs)
+    sc = scenes.make_scene(cfg)
+    g_rgb, g_depth, status = render_scene(cfg, sc)
+    assert status == 0
+    st = parity.compare_scene(oracle, cfg, scene_to_numpy(sc), range(cfg.num_obs), g_rgb, g_depth)
+    parity.assert_parity(st, name)
+
+
+@pytest.mark.parametrize("W,H", [(64, 36), (256, 144)])
+def test_sweep_resolutions_with_camera_walk(oracle, W, H):
+    from gpu_util import scene_to_numpy, upload_scene
+    B = _binding()
+    cfg = scenes.config("sweep", num_envs=2, width=W, height=H)
+    sc = scenes.make_scene(cfg)
+    batch = B.Batch(B.desc_from_config(cfg))
+    upload_scene(batch, sc)
+    rgb, depth = batch.alloc_outputs()
+    cams = sc["cams"]
+    for step in (1, 2):
+        cams = scenes.walk_cameras(cfg, sc, cams, step)
+        batch.set_cameras(cams.cuda())
+        batch.render_batch(rgb, depth)
+    assert batch.query_status() == 0
+    scn = scene_to_numpy(sc); scn["cams"] = cams.numpy()
+    st = parity.compare_scene(oracle, cfg, scn, range(cfg.num_obs), rgb.cpu().numpy(), depth.cpu().numpy())
+    parity.assert_parity(st, f"sweep {W}x{H}")
+    batch.destroy()
+
+
+def test_invariants_batching_permutation_determinism_translation():
+    from gpu_util import render_scene
+    cfg = scenes.config("rooms_boxes", num_envs=4)
+    sc = scenes.make_scene(cfg)
+    r1 = render_scene(cfg, sc)
+    r2 = render_scene(cfg, sc)
+    assert (r1[0] == r2[0]).all() and (r1[1] == r2[1]).all()                  # determinism
+    perm = torch.tensor([2, 0, 3, 1])
+    A = cfg.agents
+    sp = {k: sc[k][perm] for k in ("grid", "palette", "boxes", "box_count")}
+    sp["cams"] = sc["cams"].reshape(4, A, 6)[perm].reshape(-1, 6).contiguous()
+    rp = render_scene(cfg, sp)
+    want = r1[0].reshape(4, A, *r1[0].shape[1:])[perm.numpy()].reshape(r1[0].shape)
+    assert (rp[0] == want).all()                                              # env permutation
+    # one agent rendered alone equals the same camera inside the batch
+    cfg1 = scenes.config("rooms_boxes", num_envs=1, agents=1, movable_boxes=cfg.max_boxes, body_boxes=False)
+    e, a = 2, 3
+    s1 = {"grid": sc["grid"][e:e + 1], "palette": sc["palette"][e:e + 1], "boxes": sc["boxes"][e:e + 1],
+          "box_count": sc["box_count"][e:e + 1], "cams": sc["cams"][e * A + a: e * A + a + 1]}
+    ra = render_scene(cfg1, s1)
+    assert (ra[0][0] == r1[0][e * A + a]).all() and (ra[1][0] == r1[1][e * A + a]).all()
+
+
+def test_step_host_matches_device_path():
+    from gpu_util import upload_scene
+    B = _binding()
+    cfg = scenes.config("rooms_boxes", num_envs=12)
+    sc = scenes.make_scene(cfg)
+    batch = B.Batch(B.desc_from_config(cfg))
+    upload_scene(batch, sc)
+    batch.set_cameras(sc["cams"].cuda())
+    rgb, depth = batch.alloc_outputs()
+    batch.render_batch(rgb, depth)
+    h_rgb = torch.empty(rgb.shape, dtype=torch.uint8).pin_memory()
+    h_depth = torch.empty(depth.shape, dtype=torch.float32).pin_memory()
+    for _ in range(2):
+        batch.step_host(sc["cams"].pin_memory(), h_rgb, h_depth, boxes=sc["boxes"].contiguous(),
+                        box_count=sc["box_count"].contiguous())
+        assert torch.equal(h_rgb, rgb.cpu()) and torch.equal(h_depth, depth.cpu())
+    assert batch.query_status() == 0 and batch.launch_count() > 0
+    batch.destroy()
+
+
+def test_not_ready_and_argument_errors():
+    B = _binding()
+    cfg = scenes.config("tiny")
+    batch = B.Batch(B.desc_from_config(cfg))
+    rgb, depth = batch.alloc_outputs()
+    with pytest.raises(B.MvError) as ei:
+        batch.render_batch(rgb, depth)
+    assert ei.value.code == -4
+    sc = scenes.make_scene(cfg)
+    with pytest.raises(B.MvError) as ei:
+        batch.upload_worlds(2, 3, sc["grid"][:3].cuda(), None, None, sc["palette"][:3].cuda())
+    assert ei.value.code == -1
+    batch.upload_worlds(0, 2, sc["grid"][:2].cuda(), None, None, sc["palette"][:2].cuda())
+    batch.set_cameras(sc["cams"].cuda())
+    with pytest.raises(B.MvError) as ei:
+        batch.render_batch(rgb, depth)                  # envs 2,3 still missing
+    assert ei.value.code == -4
+    batch.upload_worlds(2, 2, sc["grid"][2:].cuda(), None, None, sc["palette"][2:].cuda())
+    batch.render_batch(rgb, depth)
+    assert batch.query_status() == 0
+    batch.destroy()
