@@ -1,0 +1,301 @@
+#!/usr/bin/env python
+"""Benchmark of the batched render step (paper Section 3.2, Eq. 2) on the headline workload:
+16384 environments x 1 agent, 128x32x128 voxel grid, 16 movable boxes, 128x72 RGB-D.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the whole per-step path: mv_set_cameras + mv_render_batch over the whole
+batch, inputs resident in HBM.  `value` is observations per second over all ranks (device time,
+CUDA events, max over ranks); `e2e` is the same metric through mv_step_host with page-locked host
+buffers (cameras and boxes copied in, frames copied out, every step).  With N > 1 (torchrun) every
+rank renders its own 16384 seeded environments: no data-path collective (weak scaling).
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+WORKLOAD = "headline"
+# DRAM bytes (read + write) per render_kernel launch from the ncu capture summarised under
+# profiles/; captured on a 2048-env slice of the same workload and scaled by 8 (traffic is
+# proportional to environments).  None until a capture exists.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peak():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi sampling in a child process for the duration of the timed region."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def cpu_oracle_rate(cfg, kept, max_seconds=25.0, max_obs=8):
+    """Observations per second of the oracle, as it stands, on this host's cores."""
+    from oracle import mv_oracle
+    mv_oracle.build()
+    desc = mv_oracle.desc_from_config(cfg)
+    done, t0 = 0, time.perf_counter()
+    for e in sorted(kept)[:max_obs]:
+        k = kept[e]
+        boxes = k["boxes"] if cfg.max_boxes > 0 else None
+        mv_oracle.render_obs(desc, k["grid"], boxes, k["box_count"], k["palette"], k["cams"][0])
+        done += 1
+        if time.perf_counter() - t0 > max_seconds:
+            break
+    dt = time.perf_counter() - t0
+    return done / dt, done, dt, mv_oracle.threads_used()
+
+
+def run_reference(args, rank):
+    """The oracle timed on a bounded sample: each step renders `sample` observations."""
+    if rank != 0:
+        return
+    import torch  # noqa: F401  (scenes use torch CPU tensors)
+    from paper_2107_08170_b200 import scenes
+    from oracle import mv_oracle
+    mv_oracle.build()
+    cfg = scenes.config(WORKLOAD)
+    sample = 2
+    n_env = sample * (args.steps + args.warmup)
+    sc = scenes.make_scene(cfg, 0, n_env)
+    desc = mv_oracle.desc_from_config(cfg)
+    g, b, c, p, cams = (sc[k].numpy() for k in ("grid", "boxes", "box_count", "palette", "cams"))
+
+    def step(i):
+        for e in range(i * sample, (i + 1) * sample):
+            mv_oracle.render_obs(desc, g[e], b[e], c[e], p[e], cams[e])
+
+    for i in range(args.warmup):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(args.warmup, args.warmup + args.steps):
+        step(i)
+    dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    cores = mv_oracle.threads_used()
+    what = f"{sample} observations of the {WORKLOAD} workload per step, all {cfg.width}x{cfg.height} pixels"
+    print(json.dumps({
+        "impl": "reference", "metric": "observations/sec", "value": value, "unit": "obs/s",
+        "grays_per_sec": value * cfg.width * cfg.height / 1e9, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg, args.gpus),
+        "cpu_baseline": {"value": value, "unit": "obs/s", "cores": cores, "kind": "oracle", "sample": what},
+        "e2e": {"value": value, "unit": "obs/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(cfg, n_gpus):
+    gx, gy, gz = cfg.grid
+    return {"workload": f"{WORKLOAD}: {cfg.num_envs} envs x {cfg.agents} agent per GPU, grid {gx}x{gy}x{gz} uint8 "
+                        f"(columns, ~15% filled), {cfg.movable_boxes} movable boxes/env, {cfg.width}x{cfg.height} RGB u8 + depth f32",
+            "envs_per_gpu": cfg.num_envs, "agents": cfg.agents, "grid": [gx, gy, gz], "boxes_per_env": cfg.max_boxes,
+            "width": cfg.width, "height": cfg.height, "parallelism": f"env-sharded x{n_gpus}, no collective",
+            "l2_policy": "inputs larger than L2 (1.1 GB of staged env blocks + 1.06 GB of frames per step vs 126 MB L2)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--envs", type=int, default=None, help="override envs per GPU (profiling small cases)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" and args.envs is None else args.warmup
+
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2107_08170_b200 import binding, scenes, workload
+
+    binding.lib()                                    # fails loudly if the CUDA library is missing
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = scenes.config(WORKLOAD) if args.envs is None else scenes.config(WORKLOAD, num_envs=args.envs)
+    keep = list(range(0, cfg.num_envs, max(cfg.num_envs // 8, 1)))[:8] if rank == 0 and not args.no_cpu else []
+    batch, cams, kept = workload.build_batch(cfg, local, env_offset=rank * cfg.num_envs, keep_envs=keep)
+    rgb, depth = batch.alloc_outputs()
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def step():
+        batch.set_cameras(cams)
+        batch.render_batch(rgb, depth)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = batch.launch_count()
+    barrier()
+    t_begin.record(stream)
+    for e0, e1, e2 in ev:
+        e0.record(stream)
+        batch.set_cameras(cams)
+        e1.record(stream)
+        batch.render_batch(rgb, depth)
+        e2.record(stream)
+    t_end.record(stream)
+    barrier()
+    total_ms = t_begin.elapsed_time(t_end)
+    launches = batch.launch_count() - launches0
+    clocks = sampler.stop()
+    render_ms = [e1.elapsed_time(e2) for _, e1, e2 in ev]
+    status = batch.query_status()
+    assert status == 0, f"device status word {status}"
+
+    # end to end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        h_cams = cams.cpu().pin_memory()
+        h_rgb = torch.empty(rgb.shape, dtype=torch.uint8).pin_memory()
+        h_depth = torch.empty(depth.shape, dtype=torch.float32).pin_memory()
+        sc_boxes = h_count = None
+        if cfg.max_boxes > 0:
+            # the boxes move every step in the simulator, so the end-to-end step re-sends them
+            sc_boxes = torch.zeros(cfg.num_envs, cfg.max_boxes, 8, dtype=torch.int32)
+            h_count = torch.zeros(cfg.num_envs, dtype=torch.int32)
+            for e0 in range(0, cfg.num_envs, 512):
+                n = min(512, cfg.num_envs - e0)
+                sc = scenes.make_scene(cfg, rank * cfg.num_envs + e0, n, device=dev)
+                sc_boxes[e0:e0 + n] = sc["boxes"].cpu(); h_count[e0:e0 + n] = sc["box_count"].cpu()
+            sc_boxes, h_count = sc_boxes.pin_memory(), h_count.pin_memory()
+        n_e2e = max(3, min(args.steps, 10))
+        for _ in range(2):
+            batch.step_host(h_cams, h_rgb, h_depth, boxes=sc_boxes, box_count=h_count)
+        barrier()
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        b0.record(stream)
+        for _ in range(n_e2e):
+            batch.step_host(h_cams, h_rgb, h_depth, boxes=sc_boxes, box_count=h_count)
+        b1.record(stream)
+        barrier()
+        e2e_ms = b0.elapsed_time(b1) / n_e2e
+        h2d = h_cams.numel() * 4 + (sc_boxes.numel() * 4 + h_count.numel() * 4 if sc_boxes is not None else 0)
+        d2h = h_rgb.numel() + h_depth.numel() * 4
+        e2e = (e2e_ms, h2d, d2h, n_e2e)
+
+    # max over ranks
+    if world > 1:
+        t = torch.tensor([total_ms, e2e[0] if e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t[0]);
+        if e2e:
+            e2e = (float(t[1]),) + e2e[1:]
+
+    if rank == 0:
+        obs_total = cfg.num_obs * world
+        ms_per_step = total_ms / args.steps
+        value = obs_total / (ms_per_step * 1e-3)
+        px = cfg.width * cfg.height
+        peak, peak_kind = measured_peak()
+        alg = workload.algorithmic_bytes(cfg)
+        k_ms = statistics.mean(render_ms)
+        achieved = alg / (k_ms * 1e-3) / 1e9
+        traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH
+        if traffic is not None and args.envs is not None:
+            traffic = traffic * cfg.num_envs / 16384
+        out = {
+            "metric": "observations/sec", "value": value, "unit": "obs/s",
+            "grays_per_sec": value * px / 1e9,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": workload_config(cfg, world),
+            "clocks": clocks, "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "kernel": "render_kernel", "achieved": achieved, "peak": peak,
+                         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": traffic, "algorithmic_bytes_per_launch": alg,
+                         "kernel_ms_mean": k_ms, "kernel_ms_min": min(render_ms), "kernel_ms_median": statistics.median(render_ms)},
+            "paper_context": "paper: 1.1e6 obs/s whole simulator on one 8x RTX 2080 Ti node (128x72 RGB, no depth)",
+        }
+        if e2e:
+            out["e2e"] = {"value": obs_total / (e2e[0] * 1e-3), "unit": "obs/s", "ms_per_step": e2e[0],
+                          "h2d_bytes_per_step": e2e[1], "d2h_bytes_per_step": e2e[2], "steps": e2e[3]}
+        if not args.no_cpu and kept:
+            rate, n, secs, cores = cpu_oracle_rate(cfg, kept)
+            out["cpu_baseline"] = {"value": rate, "unit": "obs/s", "cores": cores, "kind": "oracle",
+                                   "sample": f"{n} observations (every {max(cfg.num_envs // 8, 1)}th env) of this workload, all pixels, {secs:.1f} s"}
+        print(json.dumps(out))
+    batch.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

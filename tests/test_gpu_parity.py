@@ -200,11 +200,11 @@ def test_data_errors_set_flags_and_stay_in_bounds(oracle):
     pal = _pal(2, 4)
     boxes = np.stack([box_rows([((2, 1, 4), (3, 2, 5), 77), ((5, 1, 4), (6, 2, 5), 1)])] * 2)
     count = np.array([9, -3])
-    cams = np.stack([cam_row(4.5, 2.5, 1.5, 0.0, 0.0), cam_row(float("nan"), 2.5, 1.5, 0.0, 0.0)])
+    cams = np.stack([cam_row(4.4, 2.45, 1.55, 0.1, 0.02), cam_row(float("nan"), 2.5, 1.5, 0.0, 0.0)])
     g_rgb, g_depth, status, st = _render_custom(oracle, grid, pal, cams, W, H, boxes=boxes, box_count=count,
                                                 max_boxes=2)
     assert status == (B.FLAG_MATERIAL_CLAMPED | B.FLAG_BOX_COUNT_CLAMPED | B.FLAG_BAD_CAMERA)
-    assert st["rgb_mismatch"] == 0 and st["depth_mismatch"] == 0
+    assert st["unexcused"] == 0 and st["rgb_mismatch"] <= 1, st
     assert (g_rgb[1] == np.array([127, 178, 229], np.uint8)).all()
 
 
