@@ -5,11 +5,11 @@
 // block (1-bit occupancy grid, shaded colour table, box list) into shared memory; while it is
 // in flight the CTA clears its per-tile box masks.  Boxes are then binned to 8x4-pixel screen
 // tiles by the bounding rectangle of their projected corners (conservative, so every box that
-// a pixel's ray can touch is tested for that pixel).  Warps pull tiles from a shared counter;
-// each lane owns one pixel of the tile: it walks the occupancy grid with a 3D-DDA in shared
-// memory, tests the tile's candidate boxes with slab tests, looks the colour up in the shaded
-// table and the warp writes 24-byte RGB row segments as packed 32-bit words and 32-byte depth
-// row segments.
+// a pixel's ray can touch is tested for that pixel).  Tiles are dealt to warps round-robin;
+// each lane owns one pixel of the tile: it walks the occupancy grid with a branch-free 3D-DDA
+// in shared memory, tests the tile's candidate boxes with slab tests, looks the colour up in
+// the shaded table and the warp writes 24-byte RGB row segments as packed 32-bit words and
+// 32-byte depth row segments.
 #pragma once
 #include "mv_device.cuh"
 
@@ -45,6 +45,13 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
 }
 
 #define kInf (__int_as_float(0x7f800000))
+
+// Reciprocal to 1 ulp in one instruction; every use is inside toleranced intersection arithmetic.
+__device__ __forceinline__ float fast_rcp(float x) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
 constexpr int kWaitPolls = 1 << 18;
 
 template <int NT>
@@ -63,7 +70,6 @@ __global__ void __launch_bounds__(NT, 3) render_kernel(const RenderParams p)
     uint32_t *s_mask = reinterpret_cast<uint32_t *>(smem + p.smem_mask_off);
     float4 *s_rel = reinterpret_cast<float4 *>(smem + p.smem_rel_off);
     uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + p.smem_misc_off);
-    int *s_next = reinterpret_cast<int *>(smem + p.smem_misc_off + 8);
 
     // ---- camera record (64 bytes, same for the whole CTA)
     const float4 *cq = reinterpret_cast<const float4 *>(p.cams + obs);
@@ -85,10 +91,7 @@ __global__ void __launch_bounds__(NT, 3) render_kernel(const RenderParams p)
     }
 
     // ---- stage the environment block
-    if (tid == 0) {
-        mbar_init(s_bar, 1);
-        *s_next = 0;
-    }
+    if (tid == 0) mbar_init(s_bar, 1);
     __syncthreads();
     if (tid == 0) {
         mbar_expect_tx(s_bar, p.lay.block_bytes);
@@ -152,6 +155,7 @@ __global__ void __launch_bounds__(NT, 3) render_kernel(const RenderParams p)
 
     // ---- per-observation DDA set-up (uniform across the CTA)
     const int nvox = gx * gy * gz;
+    const unsigned last_word = (unsigned)(nvox >> 5) - 1u;
     const int stride_z = gx, stride_y = gx * gz;
     const bool cam_in = (Px >= 0.0f) && (Px < (float)gx) && (Py >= 0.0f) && (Py < (float)gy) &&
                         (Pz >= 0.0f) && (Pz < (float)gz);
@@ -159,97 +163,163 @@ __global__ void __launch_bounds__(NT, 3) render_kernel(const RenderParams p)
     if (cam_in) { cx0 = (int)floorf(Px); cy0 = (int)floorf(Py); cz0 = (int)floorf(Pz); }
     const int vi0 = cx0 + stride_z * cz0 + stride_y * cy0;
     const bool start_filled = cam_in && ((s_occ[vi0 >> 5] >> (vi0 & 31)) & 1u);
+    // distance from the eye to the two faces of its cell, and cells left before the grid ends
     const float fposx = (float)(cx0 + 1) - Px, fnegx = (float)cx0 - Px;
     const float fposy = (float)(cy0 + 1) - Py, fnegy = (float)cy0 - Py;
     const float fposz = (float)(cz0 + 1) - Pz, fnegz = (float)cz0 - Pz;
+    const float nposx = (float)(gx - 1 - cx0), nnegx = (float)cx0;
+    const float nposy = (float)(gy - 1 - cy0), nnegy = (float)cy0;
+    const float nposz = (float)(gz - 1 - cz0), nnegz = (float)cz0;
     const int max_steps = gx + gy + gz + 3;
     const uint8_t *mat_env = p.mat + (size_t)env * nvox;
     const int P_ = p.palette;
 
-    for (;;) {
-        int tile = 0;
-        if (lane == 0) tile = atomicAdd(s_next, 1);
-        tile = __shfl_sync(0xffffffffu, tile, 0);
-        if (tile >= ntiles) break;
-        const int tyi = tile / p.tiles_x, txi = tile - tyi * p.tiles_x;
-        const int px = txi * 8 + (lane & 7), py = tyi * 4 + (lane >> 3);
+    // ---- tiles: warp w takes tiles w, w + nwarps, ... (8 x 4 pixels, one per lane)
+    constexpr int kWarps = NT / 32;
+    const int warp = tid >> 5;
+    int tyi = warp / p.tiles_x, txi = warp - tyi * p.tiles_x;
+    const float lane_a = (float)(2 * (lane & 7)), lane_b = (float)(2 * (lane >> 3));
+    for (int tile = warp; tile < ntiles; tile += kWarps) {
+        // ---- ray through the pixel centre: d = F + a*Rs + b*Us, a = 2px+1-W, b = H-1-2py
+        const float a = (float)(16 * txi + 1 - W) + lane_a;
+        const float bb = (float)(H - 1 - 8 * tyi) - lane_b;
+        float dx = fmaf(bb, Ux, fmaf(a, Rx, Fx));
+        float dy = fmaf(bb, Uy, fmaf(a, Ry, Fy));
+        float dz = fmaf(bb, Uz, fmaf(a, Rz, Fz));
+        // a component that is exactly zero never crosses a cell face; 1e-30 keeps it that way
+        // without infinities in the slab arithmetic
+        dx = dx == 0.0f ? 1e-30f : dx;
+        dy = dy == 0.0f ? 1e-30f : dy;
+        dz = dz == 0.0f ? 1e-30f : dz;
+        const float ix = fast_rcp(dx), iy = fast_rcp(dy), iz = fast_rcp(dz);
+        const bool ngx = dx < 0.0f, ngy = dy < 0.0f, ngz = dz < 0.0f;
+        const float dtx = fabsf(ix), dty = fabsf(iy), dtz = fabsf(iz);
+        const int sx = ngx ? -1 : 1;
+        const int sy = ngy ? -stride_y : stride_y;
+        const int sz = ngz ? -stride_z : stride_z;
 
-        // ---- ray through the pixel centre (same fused expression as the definition)
-        const float a = (float)(2 * px + 1 - W), bb = (float)(H - 1 - 2 * py);
-        const float dx = fmaf(bb, Ux, fmaf(a, Rx, Fx));
-        const float dy = fmaf(bb, Uy, fmaf(a, Ry, Fy));
-        const float dz = fmaf(bb, Uz, fmaf(a, Rz, Fz));
-        const float ix = 1.0f / dx, iy = 1.0f / dy, iz = 1.0f / dz;
-        const bool parx = !(fabsf(ix) < kInf), pary = !(fabsf(iy) < kInf), parz = !(fabsf(iz) < kInf);
-        const float dtx = parx ? 0.0f : fabsf(ix), dty = pary ? 0.0f : fabsf(iy), dtz = parz ? 0.0f : fabsf(iz);
-        const int sx = dx >= 0.0f ? 1 : -1;
-        const int sy = dy >= 0.0f ? stride_y : -stride_y;
-        const int sz = dz >= 0.0f ? stride_z : -stride_z;
-
-        // ---- grid traversal
-        float t0x, t0y, t0z, t_exit, t_start = 0.0f;
-        int vi = vi0, axis = -1;
-        bool vhit = start_filled, alive = true;
+        // ---- grid traversal: crossing times are t0 + k*dt with integer-valued k, so the exit
+        // time below is bit-identical to the crossing that would leave the grid
+        float t0x, t0y, t0z, t_exit, t_hit = 0.0f;
+        int vi = vi0, axis0 = -1;
+        bool vhit = start_filled;
         if (cam_in) {
-            t0x = parx ? kInf : (dx >= 0.0f ? fposx : fnegx) * ix;
-            t0y = pary ? kInf : (dy >= 0.0f ? fposy : fnegy) * iy;
-            t0z = parz ? kInf : (dz >= 0.0f ? fposz : fnegz) * iz;
-            const float nx = dx >= 0.0f ? (float)(gx - 1 - cx0) : (float)cx0;
-            const float ny = dy >= 0.0f ? (float)(gy - 1 - cy0) : (float)cy0;
-            const float nz = dz >= 0.0f ? (float)(gz - 1 - cz0) : (float)cz0;
-            t_exit = fminf(fmaf(nx, dtx, t0x), fminf(fmaf(ny, dty, t0y), fmaf(nz, dtz, t0z)));
+            t0x = (ngx ? fnegx : fposx) * ix;
+            t0y = (ngy ? fnegy : fposy) * iy;
+            t0z = (ngz ? fnegz : fposz) * iz;
+            t_exit = fminf(fmaf(ngx ? nnegx : nposx, dtx, t0x),
+                           fminf(fmaf(ngy ? nnegy : nposy, dty, t0y), fmaf(ngz ? nnegz : nposz, dtz, t0z)));
         } else {
             // eye outside the grid: clip the ray to the grid's box, start in the entry cell
-            float tn = -kInf, tf = kInf;
-            const float Pc[3] = {Px, Py, Pz}, ic[3] = {ix, iy, iz}, gc[3] = {(float)gx, (float)gy, (float)gz};
-            const bool par[3] = {parx, pary, parz};
-#pragma unroll
-            for (int c = 0; c < 3; ++c) {
-                if (par[c]) {
-                    if (Pc[c] < 0.0f || Pc[c] > gc[c]) alive = false;
-                } else {
-                    const float t1 = (0.0f - Pc[c]) * ic[c], t2 = (gc[c] - Pc[c]) * ic[c];
-                    const float nr = fminf(t1, t2), fr = fmaxf(t1, t2);
-                    if (nr > tn) { tn = nr; axis = c; }
-                    tf = fminf(tf, fr);
-                }
-            }
-            if (!(tn <= tf) || !(tf > 0.0f)) alive = false;
-            if (tn < 0.0f) axis = -1;
-            t_start = fmaxf(tn, 0.0f);
-            if (!alive) t_start = 0.0f;
-            int cx = min(max((int)floorf(fmaf(t_start, dx, Px)), 0), gx - 1);
-            int cy = min(max((int)floorf(fmaf(t_start, dy, Py)), 0), gy - 1);
-            int cz = min(max((int)floorf(fmaf(t_start, dz, Pz)), 0), gz - 1);
-            if (axis == 0) cx = dx > 0.0f ? 0 : gx - 1;
-            if (axis == 1) cy = dy > 0.0f ? 0 : gy - 1;
-            if (axis == 2) cz = dz > 0.0f ? 0 : gz - 1;
+            const float x1 = (0.0f - Px) * ix, x2 = ((float)gx - Px) * ix;
+            const float y1 = (0.0f - Py) * iy, y2 = ((float)gy - Py) * iy;
+            const float z1 = (0.0f - Pz) * iz, z2 = ((float)gz - Pz) * iz;
+            const float nrx = fminf(x1, x2), nry = fminf(y1, y2), nrz = fminf(z1, z2);
+            const float tn = fmaxf(nrx, fmaxf(nry, nrz));
+            const float tf = fminf(fmaxf(x1, x2), fminf(fmaxf(y1, y2), fmaxf(z1, z2)));
+            const bool alive = (tn <= tf) && (tf > 0.0f);
+            const int eaxis = tn < 0.0f ? -1 : (nrx == tn ? 0 : (nry == tn ? 1 : 2));
+            t_hit = alive ? fmaxf(tn, 0.0f) : 0.0f;
+            int cx = min(max((int)floorf(fmaf(t_hit, dx, Px)), 0), gx - 1);
+            int cy = min(max((int)floorf(fmaf(t_hit, dy, Py)), 0), gy - 1);
+            int cz = min(max((int)floorf(fmaf(t_hit, dz, Pz)), 0), gz - 1);
+            if (eaxis == 0) cx = ngx ? gx - 1 : 0;
+            if (eaxis == 1) cy = ngy ? gy - 1 : 0;
+            if (eaxis == 2) cz = ngz ? gz - 1 : 0;
             vi = cx + stride_z * cz + stride_y * cy;
-            t0x = parx ? kInf : ((float)(cx + (dx >= 0.0f ? 1 : 0)) - Px) * ix;
-            t0y = pary ? kInf : ((float)(cy + (dy >= 0.0f ? 1 : 0)) - Py) * iy;
-            t0z = parz ? kInf : ((float)(cz + (dz >= 0.0f ? 1 : 0)) - Pz) * iz;
-            const float nx = dx >= 0.0f ? (float)(gx - 1 - cx) : (float)cx;
-            const float ny = dy >= 0.0f ? (float)(gy - 1 - cy) : (float)cy;
-            const float nz = dz >= 0.0f ? (float)(gz - 1 - cz) : (float)cz;
-            t_exit = fminf(fmaf(nx, dtx, t0x), fminf(fmaf(ny, dty, t0y), fmaf(nz, dtz, t0z)));
+            axis0 = eaxis;
+            t0x = ((float)(cx + (ngx ? 0 : 1)) - Px) * ix;
+            t0y = ((float)(cy + (ngy ? 0 : 1)) - Py) * iy;
+            t0z = ((float)(cz + (ngz ? 0 : 1)) - Pz) * iz;
+            t_exit = fminf(fmaf(ngx ? (float)cx : (float)(gx - 1 - cx), dtx, t0x),
+                           fminf(fmaf(ngy ? (float)cy : (float)(gy - 1 - cy), dty, t0y),
+                                 fmaf(ngz ? (float)cz : (float)(gz - 1 - cz), dtz, t0z)));
             vhit = alive && ((s_occ[vi >> 5] >> (vi & 31)) & 1u);
             if (!alive) t_exit = -kInf;
         }
-        float t_hit = t_start;
+        float kx = 0.0f, ky = 0.0f, kz = 0.0f;
         if (!vhit) {
-            float tx = t0x, ty = t0y, tz = t0z, kx = 0.0f, ky = 0.0f, kz = 0.0f;
-#pragma unroll 1
-            for (int it = 0; it < max_steps; ++it) {
-                const float t = fminf(tx, fminf(ty, tz));
-                if (!(t < t_exit)) break;
-                if (tx == t)      { vi += sx; kx += 1.0f; tx = fmaf(kx, dtx, t0x); axis = 0; }
-                else if (ty == t) { vi += sy; ky += 1.0f; ty = fmaf(ky, dty, t0y); axis = 1; }
-                else              { vi += sz; kz += 1.0f; tz = fmaf(kz, dtz, t0z); axis = 2; }
-                if ((unsigned)vi >= (unsigned)nvox) break;           // cannot happen; guards the read
-                if ((s_occ[vi >> 5] >> (vi & 31)) & 1u) { vhit = true; t_hit = t; break; }
-            }
+            // 3D-DDA written in PTX so that each step is a fixed short sequence of predicated
+            // instructions: t = min(tx,ty,tz); stop when t >= t_exit; step the axis whose crossing
+            // time equals t (ties: x, then y, then z): k += 1, voxel index += stride, crossing time
+            // = fma(k, dt, t0); test the voxel's occupancy bit.  The word-index clamp never binds
+            // (the exit test keeps the index inside the grid); it only guards the shared load.
+            // All loop state lives in registers declared inside the block and the outputs are
+            // written only after the last read of an input, so no operand can alias another.
+            uint32_t hit;
+            int vout;
+            float th;
+            asm volatile(
+                "{\n"
+                " .reg .pred px, py, pxy, pq;\n"
+                " .reg .f32 t, tx, ty, tz, kx, ky, kz, th;\n"
+                " .reg .u32 w, a, it, hit;\n"
+                " .reg .s32 vi;\n"
+                " mov.f32 tx, %9;\n"
+                " mov.f32 ty, %10;\n"
+                " mov.f32 tz, %11;\n"
+                " mov.f32 kx, 0f00000000;\n"
+                " mov.f32 ky, 0f00000000;\n"
+                " mov.f32 kz, 0f00000000;\n"
+                " mov.f32 th, 0f00000000;\n"
+                " mov.u32 hit, 0;\n"
+                " mov.s32 vi, %19;\n"
+                " mov.u32 it, %16;\n"
+                "MV_DDA_LOOP:\n"
+                " min.f32 t, tx, ty;\n"
+                " min.f32 t, t, tz;\n"
+                " setp.geu.f32 pq, t, %15;\n"
+                " @pq bra MV_DDA_DONE;\n"
+                " setp.eq.f32 px, tx, t;\n"
+                " setp.eq.and.f32 py, ty, t, !px;\n"
+                " or.pred pxy, px, py;\n"
+                " @px add.f32 kx, kx, 0f3F800000;\n"
+                " @px add.s32 vi, vi, %12;\n"
+                " @py add.f32 ky, ky, 0f3F800000;\n"
+                " @py add.s32 vi, vi, %13;\n"
+                " @!pxy add.f32 kz, kz, 0f3F800000;\n"
+                " @!pxy add.s32 vi, vi, %14;\n"
+                " fma.rn.f32 tx, kx, %6, %9;\n"
+                " fma.rn.f32 ty, ky, %7, %10;\n"
+                " fma.rn.f32 tz, kz, %8, %11;\n"
+                " shr.u32 a, vi, 5;\n"
+                " min.u32 a, a, %17;\n"
+                " shl.b32 a, a, 2;\n"
+                " add.u32 a, a, %18;\n"
+                " ld.shared.u32 w, [a];\n"
+                " shf.r.wrap.b32 w, w, 0, vi;\n"
+                " and.b32 w, w, 1;\n"
+                " setp.ne.u32 pq, w, 0;\n"
+                " @pq bra MV_DDA_HIT;\n"
+                " sub.u32 it, it, 1;\n"
+                " setp.ne.u32 pq, it, 0;\n"
+                " @pq bra MV_DDA_LOOP;\n"
+                " bra MV_DDA_DONE;\n"
+                "MV_DDA_HIT:\n"
+                " mov.f32 th, t;\n"
+                " mov.u32 hit, 1;\n"
+                "MV_DDA_DONE:\n"
+                " mov.f32 %0, kx;\n"
+                " mov.f32 %1, ky;\n"
+                " mov.f32 %2, kz;\n"
+                " mov.s32 %3, vi;\n"
+                " mov.f32 %4, th;\n"
+                " mov.u32 %5, hit;\n"
+                "}\n"
+                : "=f"(kx), "=f"(ky), "=f"(kz), "=r"(vout), "=f"(th), "=r"(hit)
+                : "f"(dtx), "f"(dty), "f"(dtz), "f"(t0x), "f"(t0y), "f"(t0z), "r"(sx), "r"(sy), "r"(sz),
+                  "f"(t_exit), "r"((uint32_t)max_steps), "r"(last_word), "r"(smem_addr(smem)), "r"(vi)
+                : "memory");
+            vi = vout;
+            if (hit) t_hit = th;
+            vhit = hit != 0;
         }
         __syncwarp();
+        // entered face: the axis whose crossing time equals the hit time (z, y, x order undoes the
+        // tie order of the steps); no step taken = the grid-entry axis, or none = eye inside a solid
+        int axis = axis0;
+        if (kx + ky + kz > 0.0f)
+            axis = fmaf(kz - 1.0f, dtz, t0z) == t_hit ? 2 : (fmaf(ky - 1.0f, dty, t0y) == t_hit ? 1 : 0);
 
         // ---- boxes of this tile (skip those wholly behind every lane's voxel hit)
         float tb = kInf;
@@ -296,7 +366,7 @@ __global__ void __launch_bounds__(NT, 3) render_kernel(const RenderParams p)
         }
 
         // ---- store: depth rows are 32-byte segments; RGB rows are 24 bytes = 6 packed words
-        depth_obs[(size_t)py * W + px] = depth;
+        depth_obs[(size_t)(tyi * 4 + (lane >> 3)) * W + txi * 8 + (lane & 7)] = depth;
         {
             const int r = lane / 6, j = lane - 6 * r;          // lanes 0..23: row r, word j of the row
             const int q0 = (4 * j) / 3, o = 4 * j - 3 * q0;    // first pixel and byte offset in it
@@ -310,6 +380,8 @@ __global__ void __launch_bounds__(NT, 3) render_kernel(const RenderParams p)
                 *dst = word;
             }
         }
+        txi += kWarps;
+        while (txi >= p.tiles_x) { txi -= p.tiles_x; ++tyi; }
     }
 }
 
