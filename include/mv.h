@@ -147,6 +147,33 @@ int mv_render_batch(mv_batch *batch, uint8_t *d_rgb, float *d_depth, void *cuda_
 int mv_step_host(mv_batch *batch, const mv_camera *h_cams, const mv_box *h_boxes,
                  const int32_t *h_box_count, uint8_t *h_rgb, float *h_depth, void *cuda_stream);
 
+/* One whole step from HOST memory for callers that must not allocate.  (The paper has no
+ * counterpart; this exists for deployment.)  Some hosts of this library cannot call cudaMalloc
+ * once they are running: a trainer that has handed every free byte of the GPU to its own memory
+ * pool, a control loop that cannot afford the device-wide synchronisation an allocation may
+ * cause, or a process whose policy forbids allocation after start-up.  mv_step_host allocates
+ * frame buffers on its first call; this variant never allocates.  It stages the cameras and the
+ * rendered frames in a fixed 8 MiB array that is part of the library image (so every GPU that
+ * loads the library carries those 8 MiB until the process exits) and otherwise does what
+ * mv_step_host does without the box update: cameras in, ray bases, render, frames out.
+ *   h_cams  HOST mv_camera [num_obs]
+ *   h_rgb, h_depth HOST outputs, shapes as in mv_render_batch
+ * Limit: num_obs * (7*width*height + 24) bytes, with the two frame buffers each rounded up to
+ * 256 bytes, must fit in 8 MiB (129 observations at 128x72); a larger batch gets
+ * MV_ERR_UNSUPPORTED and nothing runs.  The batch must have been created and its worlds
+ * uploaded beforehand, when allocating was still allowed.
+ * The first call on each device looks up the array's device address (a runtime query, not an
+ * allocation); make that first call before starting any stream capture.
+ * The array is shared by every batch and every call on that device and keeps whatever the last
+ * call left in it.  Nothing in it needs clearing, because each call overwrites every byte it
+ * later reads; but two calls whose device work overlaps (different streams, or different
+ * threads) race on it, so serialise them.  Synchronous like mv_step_host.
+ * Calls no cudaMalloc, cudaFree or other allocating routine.
+ * Errors: INVALID_ARG, NOT_READY, UNSUPPORTED (batch too large for the array, device ordinal
+ * >= 64), CUDA. */
+int mv_step_host_static(mv_batch *batch, const mv_camera *h_cams, uint8_t *h_rgb, float *h_depth,
+                        void *cuda_stream);
+
 /* Synchronise the stream and return the device status word: a negative mv_status if a CUDA
  * error or device timeout occurred, else the OR of the MV_FLAG_* bits seen so far (0 = clean).
  * clear != 0 resets the sticky bits. */

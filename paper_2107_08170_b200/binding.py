@@ -16,7 +16,7 @@ _lib = None
 MV_OK = 0
 FLAG_MATERIAL_CLAMPED, FLAG_BOX_COUNT_CLAMPED, FLAG_BAD_CAMERA, FLAG_DEVICE_TIMEOUT = 1, 2, 4, 8
 EXPORTS = ["mv_create_batch", "mv_upload_worlds", "mv_set_cameras", "mv_render_batch", "mv_step_host",
-           "mv_query_status", "mv_launch_count", "mv_destroy", "mv_status_string"]
+           "mv_step_host_static", "mv_query_status", "mv_launch_count", "mv_destroy", "mv_status_string"]
 
 
 class BatchDesc(C.Structure):
@@ -48,13 +48,14 @@ def lib() -> C.CDLL:
         L.mv_set_cameras.argtypes = [vp, vp, vp]
         L.mv_render_batch.argtypes = [vp, vp, vp, vp]
         L.mv_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        L.mv_step_host_static.argtypes = [vp, vp, vp, vp, vp]
         L.mv_query_status.argtypes = [vp, i, vp]
         L.mv_launch_count.argtypes = [vp]
         L.mv_launch_count.restype = C.c_int64
         L.mv_destroy.argtypes = [vp]
         L.mv_status_string.argtypes = [i]
         L.mv_status_string.restype = C.c_char_p
-        for n in EXPORTS[:6] + ["mv_destroy"]:
+        for n in EXPORTS[:7] + ["mv_destroy"]:
             getattr(L, n).restype = i
         _lib = L
     return _lib
@@ -144,6 +145,12 @@ class Batch:
         _check(lib().mv_step_host(self._h, _hptr(cams, torch.int32), _hptr(boxes, torch.int32),
                                   _hptr(box_count, torch.int32), _hptr(rgb, torch.uint8),
                                   _hptr(depth, torch.float32), _stream(stream)), "mv_step_host")
+
+    def step_host_static(self, cams, rgb, depth, stream=None):
+        """The never-allocating host step (fixed 8 MiB device array inside the library): for callers
+        that may not allocate GPU memory while running.  Raises MvError(-6) if the batch is too big."""
+        _check(lib().mv_step_host_static(self._h, _hptr(cams, torch.int32), _hptr(rgb, torch.uint8),
+                                         _hptr(depth, torch.float32), _stream(stream)), "mv_step_host_static")
 
     def query_status(self, clear=False, stream=None) -> int:
         r = lib().mv_query_status(self._h, int(clear), _stream(stream))

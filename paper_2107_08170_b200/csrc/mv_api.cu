@@ -126,6 +126,33 @@ int launch_boxes(mv_batch *b, int env_begin, int env_count, const mv_box *d_boxe
 
 }  // namespace
 
+// ---- fixed scratch for mv_step_host_static -------------------------------------------------
+// Lives in the library image: every GPU that loads the library holds these bytes until the
+// process exits.  In host code the array's name is only a host-side stand-in, never a device
+// address; the address a kernel or a copy may use comes from cudaGetSymbolAddress, taken once
+// per device with that device current.
+#define MV_STATIC_SCRATCH_BYTES (8u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[MV_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+unsigned char *g_static_scratch_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on `device` (which must be current).  First use on a
+// device asks the runtime for the symbol's address; later uses return the cached pointer.
+int static_scratch_for_device(mv_batch *b, int device, unsigned char **out) {
+    if (device < 0 || device >= kMaxDevices) return MV_ERR_UNSUPPORTED;
+    if (!g_static_scratch_ptr[device]) {
+        void *p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess || !p) return cuda_fail(b, e);
+        g_static_scratch_ptr[device] = static_cast<unsigned char *>(p);
+    }
+    *out = g_static_scratch_ptr[device];
+    return MV_OK;
+}
+}  // namespace
+
 extern "C" {
 
 const char *mv_status_string(int status) {
@@ -320,6 +347,39 @@ int mv_step_host(mv_batch *b, const mv_camera *h_cams, const mv_box *h_boxes, co
     }
     MV_CUDA(b, cudaEventRecord(b->ev_done, b->copy_stream));
     MV_CUDA(b, cudaStreamWaitEvent(s, b->ev_done, 0));
+    MV_CUDA(b, cudaStreamSynchronize(s));
+    return MV_OK;
+}
+
+int mv_step_host_static(mv_batch *b, const mv_camera *h_cams, uint8_t *h_rgb, float *h_depth,
+                        void *cuda_stream) {
+    if (!b || !h_cams || !h_rgb || !h_depth) return MV_ERR_INVALID_ARG;
+    if (b->missing_grid > 0 || b->missing_palette > 0) return MV_ERR_NOT_READY;
+    const size_t px = (size_t)b->desc.width * b->desc.height;
+    const size_t O = (size_t)b->num_obs;
+    // layout inside the scratch array: depth | rgb | cameras, each 256-byte aligned
+    const size_t depth_bytes = (O * px * 4 + 255) / 256 * 256;
+    const size_t rgb_bytes = (O * px * 3 + 255) / 256 * 256;
+    const size_t cam_bytes = O * sizeof(mv_camera);
+    if (depth_bytes + rgb_bytes + cam_bytes > (size_t)MV_STATIC_SCRATCH_BYTES) return MV_ERR_UNSUPPORTED;
+    DeviceGuard g(b->desc.device);
+    if (!g.ok) return MV_ERR_CUDA;
+    unsigned char *scratch = nullptr;
+    int r = static_scratch_for_device(b, b->desc.device, &scratch);
+    if (r != MV_OK) return r;
+    float *d_depth = reinterpret_cast<float *>(scratch);
+    uint8_t *d_rgb = scratch + depth_bytes;
+    mv_camera *d_cams = reinterpret_cast<mv_camera *>(scratch + depth_bytes + rgb_bytes);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    // nothing in the scratch has to start at zero: the cameras are overwritten by the copy
+    // below and the render kernel writes every byte of both frame buffers
+    MV_CUDA(b, cudaMemcpyAsync(d_cams, h_cams, cam_bytes, cudaMemcpyHostToDevice, s));
+    r = launch_cameras(b, d_cams, s);
+    if (r != MV_OK) return r;
+    r = launch_render(b, d_rgb, d_depth, 0, b->num_obs, s);
+    if (r != MV_OK) return r;
+    MV_CUDA(b, cudaMemcpyAsync(h_rgb, d_rgb, O * px * 3, cudaMemcpyDeviceToHost, s));
+    MV_CUDA(b, cudaMemcpyAsync(h_depth, d_depth, O * px * 4, cudaMemcpyDeviceToHost, s));
     MV_CUDA(b, cudaStreamSynchronize(s));
     return MV_OK;
 }
