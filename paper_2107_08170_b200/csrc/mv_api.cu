@@ -15,7 +15,10 @@ using namespace mv;
 
 namespace {
 
-constexpr int kRenderThreads = 256;
+#ifndef MV_NT
+#define MV_NT 384
+#endif
+constexpr int kRenderThreads = MV_NT;
 constexpr int kHostChunks = 8;
 
 inline uint32_t round_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
@@ -198,7 +201,7 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
     L.lut_off = L.occ_bytes;
     L.box_off = L.lut_off + round_up(kFaces * d.palette_size * 4, 16);
     L.count_off = L.box_off + (uint32_t)d.max_boxes * 32;
-    L.block_bytes = L.count_off + 16;
+    L.block_bytes = L.count_off + 32;
     L.stride = round_up(L.block_bytes, 128);
 
     b->tiles_x = d.width / 8;
@@ -262,6 +265,10 @@ int mv_upload_worlds(mv_batch *b, int env_begin, int env_count, const uint8_t *d
         if (blocks > 0x7fffffffull) return MV_ERR_INVALID_ARG;
         pack_grid_kernel<<<(unsigned)blocks, 256, 0, s>>>(d_grid, b->d_env_blocks, b->d_mat, b->lay, b->nvox,
                                                            env_begin, env_count, b->desc.palette_size, b->d_status);
+        b->launches++;
+        MV_CUDA(b, cudaGetLastError());
+        occupied_bounds_kernel<<<env_count, 256, 0, s>>>(b->d_env_blocks, b->lay, env_begin, b->desc.grid_x,
+                                                          b->desc.grid_y, b->desc.grid_z);
         b->launches++;
         MV_CUDA(b, cudaGetLastError());
         for (int e = env_begin; e < env_begin + env_count; ++e)

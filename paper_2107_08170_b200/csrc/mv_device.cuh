@@ -24,12 +24,13 @@ struct __align__(16) CamRec {
 static_assert(sizeof(CamRec) == 64, "CamRec must be 64 bytes");
 
 // One environment's render inputs, contiguous in HBM so that a single bulk copy stages them
-// into shared memory:  [occupancy bits | shade LUT | boxes | box count].
+// into shared memory:  [occupancy bits | shade LUT | boxes | box count + occupied bounds].
 struct EnvLayout {
     uint32_t occ_bytes;     // grid_x*grid_y*grid_z/8 rounded up to 16
     uint32_t lut_off;       // 7*palette_size RGBX words
     uint32_t box_off;       // max_boxes * 32 bytes
-    uint32_t count_off;     // 16 bytes, first int32 = box count
+    uint32_t count_off;     // 32 bytes: {box count, lo x,y,z, hi x,y,z, pad}; [lo, hi) = cell box
+                            // that contains every filled voxel (lo > hi when the grid is empty)
     uint32_t block_bytes;   // bytes staged per CTA (multiple of 16)
     uint32_t stride;        // distance between envs in HBM (multiple of 128)
 };

@@ -44,6 +44,43 @@ __global__ void pack_grid_kernel(const uint8_t *__restrict__ grid, unsigned char
     if (clamped) atomicOr(status, kFlagMaterial);
 }
 
+// Cell box [lo, hi) that contains every filled voxel of an env, from the packed occupancy bits.
+// One CTA per env; written next to the box count.  An empty grid gives lo > hi.
+__global__ void occupied_bounds_kernel(unsigned char *__restrict__ env_blocks, EnvLayout lay, int env_begin,
+                                       int gx, int gy, int gz)
+{
+    unsigned char *blk = env_blocks + (size_t)(env_begin + blockIdx.x) * lay.stride;
+    const uint32_t *occ = reinterpret_cast<const uint32_t *>(blk);
+    const int nwords = gx * gy * gz / 32;
+    int lo[3] = {gx, gy, gz}, hi[3] = {-1, -1, -1};
+    for (int w = threadIdx.x; w < nwords; w += blockDim.x) {
+        uint32_t m = occ[w];
+        while (m) {
+            const int v = w * 32 + (__ffs(m) - 1);
+            m &= m - 1;
+            const int x = v % gx, r = v / gx, z = r % gz, y = r / gz;
+            lo[0] = min(lo[0], x); hi[0] = max(hi[0], x);
+            lo[1] = min(lo[1], y); hi[1] = max(hi[1], y);
+            lo[2] = min(lo[2], z); hi[2] = max(hi[2], z);
+        }
+    }
+    __shared__ int s_lo[3], s_hi[3];
+    if (threadIdx.x < 3) { s_lo[threadIdx.x] = 1 << 30; s_hi[threadIdx.x] = -1; }
+    __syncthreads();
+#pragma unroll
+    for (int c = 0; c < 3; ++c) {
+        const int l = __reduce_min_sync(0xffffffffu, lo[c]), h = __reduce_max_sync(0xffffffffu, hi[c]);
+        if ((threadIdx.x & 31) == 0) { atomicMin(&s_lo[c], l); atomicMax(&s_hi[c], h); }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int *dst = reinterpret_cast<int *>(blk + lay.count_off);
+        dst[1] = s_lo[0]; dst[2] = s_lo[1]; dst[3] = s_lo[2];
+        dst[4] = s_hi[0] + 1; dst[5] = s_hi[1] + 1; dst[6] = s_hi[2] + 1;
+        dst[7] = 0;
+    }
+}
+
 // Shaded colour table per env: lut[face][m] = RGBX of floor(palette*I_face + 0.5), in double.
 __global__ void build_lut_kernel(const uint8_t *__restrict__ palette, unsigned char *__restrict__ env_blocks,
                                  EnvLayout lay, int env_begin, int env_count, int P,
@@ -87,7 +124,7 @@ __global__ void copy_boxes_kernel(const uint4 *__restrict__ boxes, const int32_t
     if (b == max_boxes) {
         int n = counts[e];
         if (n < 0 || n > max_boxes) { n = n < 0 ? 0 : max_boxes; atomicOr(status, kFlagBoxCount); }
-        *reinterpret_cast<int4 *>(blk + lay.count_off) = make_int4(n, 0, 0, 0);
+        *reinterpret_cast<int *>(blk + lay.count_off) = n;
         return;
     }
     uint4 lo = boxes[((size_t)e * max_boxes + b) * 2], hi = boxes[((size_t)e * max_boxes + b) * 2 + 1];

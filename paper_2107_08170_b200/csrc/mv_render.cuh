@@ -54,8 +54,39 @@ __device__ __forceinline__ float fast_rcp(float x) {
 }
 constexpr int kWaitPolls = 1 << 18;
 
+// One DDA step (see the loop in render_kernel): operands %6..%8 = dt, %9..%11 = t0, %12..%14 =
+// index strides, %15 = grid-exit time, %17 = last occupancy word, %18 = shared base address.
+#define MV_DDA_STEP                                  \
+    " min.f32 t, tx, ty, tz;\n"                      \
+    " setp.geu.f32 pq, t, %15;\n"                    \
+    " @pq bra MV_DDA_DONE;\n"                        \
+    " setp.eq.f32 px, tx, t;\n"                      \
+    " setp.eq.and.f32 py, ty, t, !px;\n"             \
+    " or.pred pxy, px, py;\n"                        \
+    " @px add.f32 kx, kx, 0f3F800000;\n"             \
+    " @px add.s32 vi, vi, %12;\n"                    \
+    " @py add.f32 ky, ky, 0f3F800000;\n"             \
+    " @py add.s32 vi, vi, %13;\n"                    \
+    " @!pxy add.f32 kz, kz, 0f3F800000;\n"           \
+    " @!pxy add.s32 vi, vi, %14;\n"                  \
+    " fma.rn.f32 tx, kx, %6, %9;\n"                  \
+    " fma.rn.f32 ty, ky, %7, %10;\n"                 \
+    " fma.rn.f32 tz, kz, %8, %11;\n"                 \
+    " shr.u32 a, vi, 5;\n"                           \
+    " min.u32 a, a, %17;\n"                          \
+    " shl.b32 a, a, 2;\n"                            \
+    " add.u32 a, a, %18;\n"                          \
+    " ld.shared.u32 w, [a];\n"                       \
+    " shf.r.wrap.b32 w, w, 0, vi;\n"                 \
+    " and.b32 w, w, 1;\n"                            \
+    " setp.ne.u32 pq, w, 0;\n"                       \
+    " @pq bra MV_DDA_HIT;\n"
+
+#ifndef MV_MINB
+#define MV_MINB 3
+#endif
 template <int NT>
-__global__ void __launch_bounds__(NT, 3) render_kernel(const RenderParams p)
+__global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, lane = tid & 31;
@@ -157,19 +188,24 @@ __global__ void __launch_bounds__(NT, 3) render_kernel(const RenderParams p)
     const int nvox = gx * gy * gz;
     const unsigned last_word = (unsigned)(nvox >> 5) - 1u;
     const int stride_z = gx, stride_y = gx * gz;
-    const bool cam_in = (Px >= 0.0f) && (Px < (float)gx) && (Py >= 0.0f) && (Py < (float)gy) &&
-                        (Pz >= 0.0f) && (Pz < (float)gz);
+    // Traversal is confined to the cell box [lo, hi) that holds every filled voxel of this env
+    // (nothing outside it can be hit), so rays that leave it, e.g. into the sky, stop there.
+    const int lox = s_count[1], loy = s_count[2], loz = s_count[3];
+    const int hix = s_count[4], hiy = s_count[5], hiz = s_count[6];
+    const bool any_voxel = (lox < hix) && (loy < hiy) && (loz < hiz);
+    const bool cam_in = any_voxel && (Px >= (float)lox) && (Px < (float)hix) && (Py >= (float)loy) &&
+                        (Py < (float)hiy) && (Pz >= (float)loz) && (Pz < (float)hiz);
     int cx0 = 0, cy0 = 0, cz0 = 0;
     if (cam_in) { cx0 = (int)floorf(Px); cy0 = (int)floorf(Py); cz0 = (int)floorf(Pz); }
     const int vi0 = cx0 + stride_z * cz0 + stride_y * cy0;
     const bool start_filled = cam_in && ((s_occ[vi0 >> 5] >> (vi0 & 31)) & 1u);
-    // distance from the eye to the two faces of its cell, and cells left before the grid ends
+    // distance from the eye to the two faces of its cell, and cells left before the box ends
     const float fposx = (float)(cx0 + 1) - Px, fnegx = (float)cx0 - Px;
     const float fposy = (float)(cy0 + 1) - Py, fnegy = (float)cy0 - Py;
     const float fposz = (float)(cz0 + 1) - Pz, fnegz = (float)cz0 - Pz;
-    const float nposx = (float)(gx - 1 - cx0), nnegx = (float)cx0;
-    const float nposy = (float)(gy - 1 - cy0), nnegy = (float)cy0;
-    const float nposz = (float)(gz - 1 - cz0), nnegz = (float)cz0;
+    const float nposx = (float)(hix - 1 - cx0), nnegx = (float)(cx0 - lox);
+    const float nposy = (float)(hiy - 1 - cy0), nnegy = (float)(cy0 - loy);
+    const float nposz = (float)(hiz - 1 - cz0), nnegz = (float)(cz0 - loz);
     const int max_steps = gx + gy + gz + 3;
     const uint8_t *mat_env = p.mat + (size_t)env * nvox;
     const int P_ = p.palette;
@@ -210,30 +246,31 @@ __global__ void __launch_bounds__(NT, 3) render_kernel(const RenderParams p)
             t_exit = fminf(fmaf(ngx ? nnegx : nposx, dtx, t0x),
                            fminf(fmaf(ngy ? nnegy : nposy, dty, t0y), fmaf(ngz ? nnegz : nposz, dtz, t0z)));
         } else {
-            // eye outside the grid: clip the ray to the grid's box, start in the entry cell
-            const float x1 = (0.0f - Px) * ix, x2 = ((float)gx - Px) * ix;
-            const float y1 = (0.0f - Py) * iy, y2 = ((float)gy - Py) * iy;
-            const float z1 = (0.0f - Pz) * iz, z2 = ((float)gz - Pz) * iz;
+            // eye outside the occupied box: clip the ray to it, start in the entry cell
+            const float x1 = ((float)lox - Px) * ix, x2 = ((float)hix - Px) * ix;
+            const float y1 = ((float)loy - Py) * iy, y2 = ((float)hiy - Py) * iy;
+            const float z1 = ((float)loz - Pz) * iz, z2 = ((float)hiz - Pz) * iz;
             const float nrx = fminf(x1, x2), nry = fminf(y1, y2), nrz = fminf(z1, z2);
             const float tn = fmaxf(nrx, fmaxf(nry, nrz));
             const float tf = fminf(fmaxf(x1, x2), fminf(fmaxf(y1, y2), fmaxf(z1, z2)));
-            const bool alive = (tn <= tf) && (tf > 0.0f);
+            const bool alive = any_voxel && (tn <= tf) && (tf > 0.0f);
             const int eaxis = tn < 0.0f ? -1 : (nrx == tn ? 0 : (nry == tn ? 1 : 2));
             t_hit = alive ? fmaxf(tn, 0.0f) : 0.0f;
-            int cx = min(max((int)floorf(fmaf(t_hit, dx, Px)), 0), gx - 1);
-            int cy = min(max((int)floorf(fmaf(t_hit, dy, Py)), 0), gy - 1);
-            int cz = min(max((int)floorf(fmaf(t_hit, dz, Pz)), 0), gz - 1);
-            if (eaxis == 0) cx = ngx ? gx - 1 : 0;
-            if (eaxis == 1) cy = ngy ? gy - 1 : 0;
-            if (eaxis == 2) cz = ngz ? gz - 1 : 0;
+            int cx = min(max((int)floorf(fmaf(t_hit, dx, Px)), lox), hix - 1);
+            int cy = min(max((int)floorf(fmaf(t_hit, dy, Py)), loy), hiy - 1);
+            int cz = min(max((int)floorf(fmaf(t_hit, dz, Pz)), loz), hiz - 1);
+            if (eaxis == 0) cx = ngx ? hix - 1 : lox;
+            if (eaxis == 1) cy = ngy ? hiy - 1 : loy;
+            if (eaxis == 2) cz = ngz ? hiz - 1 : loz;
+            if (!alive) { cx = cy = cz = 0; }
             vi = cx + stride_z * cz + stride_y * cy;
             axis0 = eaxis;
             t0x = ((float)(cx + (ngx ? 0 : 1)) - Px) * ix;
             t0y = ((float)(cy + (ngy ? 0 : 1)) - Py) * iy;
             t0z = ((float)(cz + (ngz ? 0 : 1)) - Pz) * iz;
-            t_exit = fminf(fmaf(ngx ? (float)cx : (float)(gx - 1 - cx), dtx, t0x),
-                           fminf(fmaf(ngy ? (float)cy : (float)(gy - 1 - cy), dty, t0y),
-                                 fmaf(ngz ? (float)cz : (float)(gz - 1 - cz), dtz, t0z)));
+            t_exit = fminf(fmaf(ngx ? (float)(cx - lox) : (float)(hix - 1 - cx), dtx, t0x),
+                           fminf(fmaf(ngy ? (float)(cy - loy) : (float)(hiy - 1 - cy), dty, t0y),
+                                 fmaf(ngz ? (float)(cz - loz) : (float)(hiz - 1 - cz), dtz, t0z)));
             vhit = alive && ((s_occ[vi >> 5] >> (vi & 31)) & 1u);
             if (!alive) t_exit = -kInf;
         }
@@ -242,8 +279,9 @@ __global__ void __launch_bounds__(NT, 3) render_kernel(const RenderParams p)
             // 3D-DDA written in PTX so that each step is a fixed short sequence of predicated
             // instructions: t = min(tx,ty,tz); stop when t >= t_exit; step the axis whose crossing
             // time equals t (ties: x, then y, then z): k += 1, voxel index += stride, crossing time
-            // = fma(k, dt, t0); test the voxel's occupancy bit.  The word-index clamp never binds
-            // (the exit test keeps the index inside the grid); it only guards the shared load.
+            // = fma(k, dt, t0); test the voxel's occupancy bit.  Two steps per trip of the bounded
+            // loop.  The word-index clamp never binds (the exit test keeps the index inside the
+            // grid); it only guards the shared load.
             // All loop state lives in registers declared inside the block and the outputs are
             // written only after the last read of an input, so no operand can alias another.
             uint32_t hit;
@@ -253,8 +291,8 @@ __global__ void __launch_bounds__(NT, 3) render_kernel(const RenderParams p)
                 "{\n"
                 " .reg .pred px, py, pxy, pq;\n"
                 " .reg .f32 t, tx, ty, tz, kx, ky, kz, th;\n"
-                " .reg .u32 w, a, it, hit;\n"
-                " .reg .s32 vi;\n"
+                " .reg .u32 w, a, hit;\n"
+                " .reg .s32 vi, it;\n"
                 " mov.f32 tx, %9;\n"
                 " mov.f32 ty, %10;\n"
                 " mov.f32 tz, %11;\n"
@@ -264,35 +302,12 @@ __global__ void __launch_bounds__(NT, 3) render_kernel(const RenderParams p)
                 " mov.f32 th, 0f00000000;\n"
                 " mov.u32 hit, 0;\n"
                 " mov.s32 vi, %19;\n"
-                " mov.u32 it, %16;\n"
+                " mov.s32 it, %16;\n"
                 "MV_DDA_LOOP:\n"
-                " min.f32 t, tx, ty;\n"
-                " min.f32 t, t, tz;\n"
-                " setp.geu.f32 pq, t, %15;\n"
-                " @pq bra MV_DDA_DONE;\n"
-                " setp.eq.f32 px, tx, t;\n"
-                " setp.eq.and.f32 py, ty, t, !px;\n"
-                " or.pred pxy, px, py;\n"
-                " @px add.f32 kx, kx, 0f3F800000;\n"
-                " @px add.s32 vi, vi, %12;\n"
-                " @py add.f32 ky, ky, 0f3F800000;\n"
-                " @py add.s32 vi, vi, %13;\n"
-                " @!pxy add.f32 kz, kz, 0f3F800000;\n"
-                " @!pxy add.s32 vi, vi, %14;\n"
-                " fma.rn.f32 tx, kx, %6, %9;\n"
-                " fma.rn.f32 ty, ky, %7, %10;\n"
-                " fma.rn.f32 tz, kz, %8, %11;\n"
-                " shr.u32 a, vi, 5;\n"
-                " min.u32 a, a, %17;\n"
-                " shl.b32 a, a, 2;\n"
-                " add.u32 a, a, %18;\n"
-                " ld.shared.u32 w, [a];\n"
-                " shf.r.wrap.b32 w, w, 0, vi;\n"
-                " and.b32 w, w, 1;\n"
-                " setp.ne.u32 pq, w, 0;\n"
-                " @pq bra MV_DDA_HIT;\n"
-                " sub.u32 it, it, 1;\n"
-                " setp.ne.u32 pq, it, 0;\n"
+                MV_DDA_STEP
+                MV_DDA_STEP
+                " sub.u32 it, it, 2;\n"
+                " setp.gt.s32 pq, it, 0;\n"
                 " @pq bra MV_DDA_LOOP;\n"
                 " bra MV_DDA_DONE;\n"
                 "MV_DDA_HIT:\n"
