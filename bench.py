@@ -27,10 +27,9 @@ ROOT = Path(__file__).resolve().parent
 sys.path.insert(0, str(ROOT))
 
 WORKLOAD = "headline"
-# DRAM bytes (read + write) per render_kernel launch from the ncu capture summarised under
-# profiles/; captured on a 2048-env slice of the same workload and scaled by 8 (traffic is
-# proportional to environments).  None until a capture exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM bytes (read 1.24 GB + write 1.01 GB) of one render_kernel launch on this full workload, from
+# the one-pass ncu capture summarised in profiles/render_kernel_headline_launch_list.md.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 2.25e9
 
 
 def measured_peak():
