@@ -187,7 +187,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2107_08170_b200 import binding, scenes, workload
+    from paper_2107_08170_b200 import binding, scenes, shard, workload
 
     binding.lib()                                    # fails loudly if the CUDA library is missing
     assert torch.cuda.is_available(), "bench.py needs a CUDA device"
@@ -198,7 +198,7 @@ def main():
 
     cfg = scenes.config(WORKLOAD) if args.envs is None else scenes.config(WORKLOAD, num_envs=args.envs)
     keep = list(range(0, cfg.num_envs, max(cfg.num_envs // 8, 1)))[:8] if rank == 0 and not args.no_cpu else []
-    batch, cams, kept = workload.build_batch(cfg, local, env_offset=rank * cfg.num_envs, keep_envs=keep)
+    batch, cams, kept = workload.build_batch(cfg, local, env_offset=shard.env_offset(rank, cfg.num_envs), keep_envs=keep)
     rgb, depth = batch.alloc_outputs()
     stream = torch.cuda.current_stream()
 
@@ -268,12 +268,10 @@ def main():
         e2e = (e2e_ms, h2d, d2h, n_e2e)
 
     # max over ranks
-    if world > 1:
-        t = torch.tensor([total_ms, e2e[0] if e2e else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t[0]);
-        if e2e:
-            e2e = (float(t[1]),) + e2e[1:]
+    mx = shard.max_over_ranks([total_ms, e2e[0] if e2e else 0.0], dev)
+    total_ms = mx[0]
+    if e2e:
+        e2e = (mx[1],) + e2e[1:]
 
     if rank == 0:
         obs_total = cfg.num_obs * world
