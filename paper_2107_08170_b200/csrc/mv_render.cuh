@@ -215,6 +215,15 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     const int warp = tid >> 5;
     int tyi = warp / p.tiles_x, txi = warp - tyi * p.tiles_x;
     const float lane_a = (float)(2 * (lane & 7)), lane_b = (float)(2 * (lane >> 3));
+    // store plan, fixed per lane: depth goes to the lane's own pixel; lanes 0..23 each write one
+    // 32-bit word (row r, word j) of the tile's four 24-byte RGB row segments, assembled from the
+    // packed colours of pixels q0 and q0+1 of that row
+    const int st_r = lane / 6, st_j = lane - 6 * st_r;
+    const int st_q0 = (4 * st_j) / 3, st_shift = 8 * (4 * st_j - 3 * st_q0);
+    const int st_src = (st_r & 3) * 8 + st_q0;
+    const int depth_lane_off = (lane >> 3) * W + (lane & 7);
+    const int rgb_lane_off = st_r * W * 3 + st_j * 4;
+    int tile_px = (tyi * 4) * W + txi * 8;          // first pixel of the warp's current tile
     for (int tile = warp; tile < ntiles; tile += kWarps) {
         // ---- ray through the pixel centre: d = F + a*Rs + b*Us, a = 2px+1-W, b = H-1-2py
         const float a = (float)(16 * txi + 1 - W) + lane_a;
@@ -275,6 +284,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             if (!alive) t_exit = -kInf;
         }
         float kx = 0.0f, ky = 0.0f, kz = 0.0f;
+        bool loop_hit = false;
         if (!vhit) {
             // 3D-DDA written in PTX so that each step is a fixed short sequence of predicated
             // instructions: t = min(tx,ty,tz); stop when t >= t_exit; step the axis whose crossing
@@ -327,13 +337,13 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                 : "memory");
             vi = vout;
             if (hit) t_hit = th;
-            vhit = hit != 0;
+            vhit = loop_hit = hit != 0;
         }
         __syncwarp();
         // entered face: the axis whose crossing time equals the hit time (z, y, x order undoes the
         // tie order of the steps); no step taken = the grid-entry axis, or none = eye inside a solid
         int axis = axis0;
-        if (kx + ky + kz > 0.0f)
+        if (loop_hit)
             axis = fmaf(kz - 1.0f, dtz, t0z) == t_hit ? 2 : (fmaf(ky - 1.0f, dty, t0y) == t_hit ? 1 : 0);
 
         // ---- boxes of this tile (skip those wholly behind every lane's voxel hit)
@@ -381,22 +391,16 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         }
 
         // ---- store: depth rows are 32-byte segments; RGB rows are 24 bytes = 6 packed words
-        depth_obs[(size_t)(tyi * 4 + (lane >> 3)) * W + txi * 8 + (lane & 7)] = depth;
+        depth_obs[tile_px + depth_lane_off] = depth;
         {
-            const int r = lane / 6, j = lane - 6 * r;          // lanes 0..23: row r, word j of the row
-            const int q0 = (4 * j) / 3, o = 4 * j - 3 * q0;    // first pixel and byte offset in it
-            const int src = (r & 3) * 8 + q0;
-            const uint32_t ca = __shfl_sync(0xffffffffu, rgbx, src);
-            const uint32_t cb = __shfl_sync(0xffffffffu, rgbx, (src + 1) & 31);
-            const uint32_t lo = (ca & 0xffffffu) | (cb << 24), hi = (cb & 0xffffffu) >> 8;
-            const uint32_t word = __funnelshift_r(lo, hi, 8 * o);
-            if (lane < 24) {
-                uint32_t *dst = reinterpret_cast<uint32_t *>(rgb_obs + ((size_t)(tyi * 4 + r) * W + txi * 8) * 3) + j;
-                *dst = word;
-            }
+            const uint32_t ca = __shfl_sync(0xffffffffu, rgbx, st_src);
+            const uint32_t cb = __shfl_sync(0xffffffffu, rgbx, (st_src + 1) & 31);
+            const uint32_t word = __funnelshift_r(ca | (cb << 24), cb >> 8, st_shift);
+            if (lane < 24) *reinterpret_cast<uint32_t *>(rgb_obs + (tile_px * 3 + rgb_lane_off)) = word;
         }
         txi += kWarps;
-        while (txi >= p.tiles_x) { txi -= p.tiles_x; ++tyi; }
+        tile_px += 8 * kWarps;
+        while (txi >= p.tiles_x) { txi -= p.tiles_x; ++tyi; tile_px += 3 * W; }
     }
 }
 
