@@ -264,3 +264,74 @@ int mvo_render_obs(const mvo_desc *D, const uint8_t *grid, const mvo_box *boxes,
     free(pxy);
     return r;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Pixel-space GUI overlay (paper Appendix A.2: geometric primitives drawn in the agent's field
+ * of view, e.g. the time-left bar).  Reading: a short list of axis-aligned filled rectangles in
+ * pixel coordinates, half-open [x0,x1) x [y0,y1), clipped to the image, painted over the RGB
+ * frame in list order (later rectangles on top); the depth channel is not touched.
+ * Record layout (16 bytes): int16 x0, y0, x1, y1; uint8 r, g, b, pad; uint32 pad. */
+typedef struct { int16_t x0, y0, x1, y1; uint8_t rgb[3]; uint8_t pad0; uint32_t pad1; } mvo_rect;
+
+void mvo_overlay(int W, int H, const mvo_rect *rects, int count, uint8_t *rgb)
+{
+    for (int r = 0; r < count; ++r)
+        for (int y = 0; y < H; ++y)
+            for (int x = 0; x < W; ++x)
+                if (x >= rects[r].x0 && x < rects[r].x1 && y >= rects[r].y0 && y < rects[r].y1) {
+                    rgb[(y * W + x) * 3] = rects[r].rgb[0];
+                    rgb[(y * W + x) * 3 + 1] = rects[r].rgb[1];
+                    rgb[(y * W + x) * 3 + 2] = rects[r].rgb[2];
+                }
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Agent motion with collision against the voxel grid (paper Section 3.1: movement and collision
+ * checking for agents are continuous; Section 3.2, Eq. 1: S' = Physics(S, A), here only the
+ * agent-body part of it).  Reading, since the paper gives no formula:
+ *   yaw' = yaw + dyaw; pitch' = clamp(pitch + dpitch, -max_pitch, max_pitch)      (float)
+ *   step = forward*(sin yaw', 0, cos yaw') + strafe*(cos yaw', 0, -sin yaw')      (double)
+ *   x_try = (float)(x + step.x), z_try = (float)(z + step.z)
+ *   the body is the box [x-hw, x+hw] x [y-below, y+above] x [z-hw, z+hw] (float arithmetic);
+ *   the x move is kept iff the body at (x_try, y, z) lies inside the grid and touches no filled
+ *   voxel; then the z move is tried the same way from the accepted x (axis-separated sliding).
+ *   Cells touched along an axis: floor(lo) .. floor(hi), both ends included.
+ * cam = {x, y, z, yaw, pitch} in/out; move = {forward, strafe, dyaw, dpitch};
+ * shape = {hw, below, above}.  Returns bit 0 = x move kept, bit 1 = z move kept. */
+static int body_free(const uint8_t *grid, int gx, int gy, int gz, float x, float y, float z,
+                     const float shape[3])
+{
+    float lo[3] = { x - shape[0], y - shape[1], z - shape[0] };
+    float hi[3] = { x + shape[0], y + shape[2], z + shape[0] };
+    int g[3] = { gx, gy, gz }, c0[3], c1[3];
+    for (int c = 0; c < 3; ++c) {
+        if (!(lo[c] >= 0.0f) || !(hi[c] < (float)g[c])) return 0;      /* also rejects NaN */
+        c0[c] = (int)floorf(lo[c]);
+        c1[c] = (int)floorf(hi[c]);
+    }
+    for (int j = c0[1]; j <= c1[1]; ++j)
+        for (int k = c0[2]; k <= c1[2]; ++k)
+            for (int i = c0[0]; i <= c1[0]; ++i)
+                if (grid[((size_t)j * gz + k) * gx + i]) return 0;
+    return 1;
+}
+
+int mvo_move_agent(const uint8_t *grid, int gx, int gy, int gz, float cam[5], const float move[4],
+                   const float shape[3], float max_pitch)
+{
+    float yaw = cam[3] + move[2];
+    float pitch = cam[4] + move[3];
+    if (pitch > max_pitch) pitch = max_pitch;
+    if (pitch < -max_pitch) pitch = -max_pitch;
+    double sy = sin((double)yaw), cy = cos((double)yaw);
+    double sxd = (double)move[0] * sy + (double)move[1] * cy;
+    double szd = (double)move[0] * cy - (double)move[1] * sy;
+    float x_try = (float)((double)cam[0] + sxd);
+    float z_try = (float)((double)cam[2] + szd);
+    int kept = 0;
+    float x = cam[0], z = cam[2];
+    if (body_free(grid, gx, gy, gz, x_try, cam[1], z, shape)) { x = x_try; kept |= 1; }
+    if (body_free(grid, gx, gy, gz, x, cam[1], z_try, shape)) { z = z_try; kept |= 2; }
+    cam[0] = x; cam[2] = z; cam[3] = yaw; cam[4] = pitch;
+    return kept;
+}

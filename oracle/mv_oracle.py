@@ -144,3 +144,32 @@ def render_scene(cfg, scene: dict, obs_indices=None):
         out.append(render_obs(desc, grid[e], b, count[e], palette[e], cams[o]))
     rgb = np.stack([x[0] for x in out]); depth = np.stack([x[1] for x in out]); ids = np.stack([x[2] for x in out])
     return rgb, depth, ids
+
+
+RECT_DTYPE = np.dtype([("x0", "<i2"), ("y0", "<i2"), ("x1", "<i2"), ("y1", "<i2"),
+                       ("rgb", "u1", (3,)), ("pad0", "u1"), ("pad1", "<u4")])
+assert RECT_DTYPE.itemsize == 16
+
+
+def overlay(rgb, rects, count):
+    """Paint `count` rectangles (RECT_DTYPE records) over one frame rgb[H][W][3], in place."""
+    H, W, _ = rgb.shape
+    rects = np.ascontiguousarray(rects, dtype=RECT_DTYPE)
+    assert rgb.flags["C_CONTIGUOUS"] and rgb.dtype == np.uint8
+    lib().mvo_overlay(C.c_int(W), C.c_int(H), rects.ctypes.data_as(C.c_void_p), C.c_int(int(count)),
+                      rgb.ctypes.data_as(C.c_void_p))
+    return rgb
+
+
+def move_agent(grid, cam5, move4, shape3=(0.25, 0.75, 0.25), max_pitch=1.0):
+    """One agent: cam5 = float32 (x,y,z,yaw,pitch) -> (new cam5, kept bits)."""
+    grid = np.ascontiguousarray(grid, dtype=np.uint8)
+    gy, gz, gx = grid.shape
+    cam = np.array(cam5, dtype=np.float32).copy()
+    move = np.array(move4, dtype=np.float32)
+    shape = np.array(shape3, dtype=np.float32)
+    L = lib()
+    L.mvo_move_agent.restype = C.c_int
+    kept = L.mvo_move_agent(_ptr(grid, C.c_uint8), C.c_int(gx), C.c_int(gy), C.c_int(gz), _ptr(cam, C.c_float),
+                            _ptr(move, C.c_float), _ptr(shape, C.c_float), C.c_float(float(np.float32(max_pitch))))
+    return cam, kept
