@@ -81,6 +81,30 @@ typedef struct mv_camera {
     int32_t self_box;
 } mv_camera;
 
+/* One filled rectangle of the pixel-space GUI (paper Appendix A.2: bars and indicators drawn in
+ * the agent's field of view, e.g. the time-left bar).  Pixel coordinates, half-open
+ * [x0,x1) x [y0,y1), clipped to the image.  16 bytes. */
+typedef struct mv_overlay_rect {
+    int16_t x0, y0, x1, y1;
+    uint8_t rgb[3];
+    uint8_t pad0;
+    uint32_t pad1;
+} mv_overlay_rect;
+
+/* One agent's motion command for a step (paper Appendix A.2, action table: moving, strafing,
+ * turning, vertical gaze), already scaled to world units and radians.  16 bytes. */
+typedef struct mv_agent_move {
+    float forward, strafe;              /* along the horizontal view direction / to the right */
+    float dyaw, dpitch;
+} mv_agent_move;
+
+/* Agent body used for collision: the box [x-half_width, x+half_width] x
+ * [y-below_eye, y+above_eye] x [z-half_width, z+half_width] around the eye. */
+typedef struct mv_body_shape {
+    float half_width, below_eye, above_eye;
+    float max_pitch;                    /* |pitch| is clamped to this */
+} mv_body_shape;
+
 typedef struct mv_batch_desc {
     int32_t num_envs;                   /* N >= 1 */
     int32_t agents_per_env;             /* M >= 1 */
@@ -97,6 +121,7 @@ typedef struct mv_batch_desc {
     uint8_t pad;
     float miss_depth;
     int32_t device;                     /* CUDA device ordinal */
+    int32_t max_overlay_rects;          /* GUI rectangles per observation, 0..16 (0 = no overlay) */
 } mv_batch_desc;
 
 /* Allocate the device-resident world store, camera table and status word for a batch
@@ -132,6 +157,33 @@ int mv_set_cameras(mv_batch *batch, const mv_camera *d_cams, void *cuda_stream);
  *   d_depth DEVICE float [num_obs][height][width]
  * Errors: INVALID_ARG, NOT_READY (some env has no grid/palette yet, or no cameras), CUDA. */
 int mv_render_batch(mv_batch *batch, uint8_t *d_rgb, float *d_depth, void *cuda_stream);
+
+/* Set the GUI overlay of every observation (paper Appendix A.2).  The rectangles are painted
+ * over the RGB frame in list order (later ones on top) by the render kernel's store stage; depth
+ * is not touched.  The overlay stays in force until set again.
+ *   d_rects DEVICE mv_overlay_rect [num_obs][max_overlay_rects], or NULL to clear all overlays
+ *   d_count DEVICE int32 [num_obs] rectangles in use per observation (clamped to
+ *           0..max_overlay_rects); required when d_rects is given
+ * Errors: INVALID_ARG (d_rects without d_count, or the batch was created with
+ * max_overlay_rects == 0 and d_rects is not NULL), CUDA. */
+int mv_set_overlays(mv_batch *batch, const mv_overlay_rect *d_rects, const int32_t *d_count,
+                    void *cuda_stream);
+
+/* Move every agent and collide its body with the voxel grid (paper Section 3.1: agent movement
+ * and collision checking are continuous; Section 3.2, Eq. 1, the agent part of
+ * S' = Physics(S, A)), then rebuild its ray basis, so that mv_render_batch can follow directly.
+ * Per agent: yaw += dyaw; pitch = clamp(pitch + dpitch); the horizontal step
+ * forward*(sin yaw, cos yaw) + strafe*(cos yaw, -sin yaw) is evaluated in double and added to the
+ * float position; the x move is kept iff the body at the new x lies inside the grid and touches
+ * no filled voxel, then the z move likewise from the accepted x (axis-separated sliding).  Movable
+ * boxes do not block.  If the camera's self_box is a valid box index, that box is moved with the
+ * body (material kept) so that other agents see it.
+ *   d_cams_inout DEVICE mv_camera [num_obs], updated in place (the caller owns agent state)
+ *   d_moves      DEVICE mv_agent_move [num_obs]
+ *   shape        HOST pointer, or NULL for {0.25, 0.75, 0.25, max_pitch 1.0}
+ * Needs the grids of all envs (NOT_READY otherwise).  Errors: INVALID_ARG, NOT_READY, CUDA. */
+int mv_move_agents(mv_batch *batch, mv_camera *d_cams_inout, const mv_agent_move *d_moves,
+                   const mv_body_shape *shape, void *cuda_stream);
 
 /* One whole step from HOST memory (paper Section 3.2: by default the rendered frames are
  * transferred to CPU memory): copies cameras (and, if given, this step's boxes) host->device,

@@ -16,7 +16,7 @@ _lib = None
 MV_OK = 0
 FLAG_MATERIAL_CLAMPED, FLAG_BOX_COUNT_CLAMPED, FLAG_BAD_CAMERA, FLAG_DEVICE_TIMEOUT = 1, 2, 4, 8
 EXPORTS = ["mv_create_batch", "mv_upload_worlds", "mv_set_cameras", "mv_render_batch", "mv_step_host",
-           "mv_step_host_static", "mv_query_status", "mv_launch_count", "mv_destroy", "mv_status_string"]
+           "mv_step_host_static", "mv_set_overlays", "mv_move_agents", "mv_query_status", "mv_launch_count", "mv_destroy", "mv_status_string"]
 
 
 class BatchDesc(C.Structure):
@@ -25,7 +25,7 @@ class BatchDesc(C.Structure):
                 ("max_boxes", C.c_int32), ("width", C.c_int32), ("height", C.c_int32),
                 ("palette_size", C.c_int32), ("hfov_rad", C.c_float), ("light_dir", C.c_float * 3),
                 ("ambient", C.c_float), ("sky_rgb", C.c_uint8 * 3), ("pad", C.c_uint8),
-                ("miss_depth", C.c_float), ("device", C.c_int32)]
+                ("miss_depth", C.c_float), ("device", C.c_int32), ("max_overlay_rects", C.c_int32)]
 
 
 class MvError(RuntimeError):
@@ -49,13 +49,15 @@ def lib() -> C.CDLL:
         L.mv_render_batch.argtypes = [vp, vp, vp, vp]
         L.mv_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.mv_step_host_static.argtypes = [vp, vp, vp, vp, vp]
+        L.mv_set_overlays.argtypes = [vp, vp, vp, vp]
+        L.mv_move_agents.argtypes = [vp, vp, vp, vp, vp]
         L.mv_query_status.argtypes = [vp, i, vp]
         L.mv_launch_count.argtypes = [vp]
         L.mv_launch_count.restype = C.c_int64
         L.mv_destroy.argtypes = [vp]
         L.mv_status_string.argtypes = [i]
         L.mv_status_string.restype = C.c_char_p
-        for n in EXPORTS[:7] + ["mv_destroy"]:
+        for n in EXPORTS[:9] + ["mv_destroy"]:
             getattr(L, n).restype = i
         _lib = L
     return _lib
@@ -72,7 +74,7 @@ def _check(code: int, where: str):
 
 def make_desc(num_envs, agents_per_env, grid, max_boxes, width, height, palette_size, hfov_rad=None,
               light_dir=(0.36, 0.80, 0.48), ambient=0.3, sky_rgb=(127, 178, 229), miss_depth=0.0,
-              device=0) -> BatchDesc:
+              device=0, max_overlay_rects=0) -> BatchDesc:
     import math
     d = BatchDesc()
     d.num_envs, d.agents_per_env = num_envs, agents_per_env
@@ -84,13 +86,19 @@ def make_desc(num_envs, agents_per_env, grid, max_boxes, width, height, palette_
     d.sky_rgb = (C.c_uint8 * 3)(*sky_rgb)
     d.miss_depth = miss_depth
     d.device = device
+    d.max_overlay_rects = max_overlay_rects
     return d
 
 
-def desc_from_config(cfg, device=0) -> BatchDesc:
+class BodyShape(C.Structure):
+    _fields_ = [("half_width", C.c_float), ("below_eye", C.c_float), ("above_eye", C.c_float),
+                ("max_pitch", C.c_float)]
+
+
+def desc_from_config(cfg, device=0, max_overlay_rects=0) -> BatchDesc:
     return make_desc(cfg.num_envs, cfg.agents, cfg.grid, cfg.max_boxes, cfg.width, cfg.height,
                      cfg.palette_size, cfg.hfov_rad, cfg.light_dir, cfg.ambient, cfg.sky_rgb,
-                     cfg.miss_depth, device)
+                     cfg.miss_depth, device, max_overlay_rects)
 
 
 def _dptr(t, dtype=None):
@@ -145,6 +153,19 @@ class Batch:
         _check(lib().mv_step_host(self._h, _hptr(cams, torch.int32), _hptr(boxes, torch.int32),
                                   _hptr(box_count, torch.int32), _hptr(rgb, torch.uint8),
                                   _hptr(depth, torch.float32), _stream(stream)), "mv_step_host")
+
+    def set_overlays(self, rects=None, count=None, stream=None):
+        """rects: CUDA int32 [num_obs][max_overlay_rects][4] (the 16-byte records viewed as int32), or None."""
+        _check(lib().mv_set_overlays(self._h, _dptr(rects, torch.int32), _dptr(count, torch.int32),
+                                     _stream(stream)), "mv_set_overlays")
+
+    def move_agents(self, cams, moves, shape=None, stream=None):
+        """cams: CUDA int32 [num_obs][6], updated in place; moves: CUDA float32 [num_obs][4]."""
+        sp = None
+        if shape is not None:
+            sp = C.byref(BodyShape(*shape))
+        _check(lib().mv_move_agents(self._h, _dptr(cams, torch.int32), _dptr(moves, torch.float32), sp,
+                                    _stream(stream)), "mv_move_agents")
 
     def step_host_static(self, cams, rgb, depth, stream=None):
         """The never-allocating host step (fixed 8 MiB device array inside the library): for callers

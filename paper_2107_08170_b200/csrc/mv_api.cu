@@ -34,6 +34,9 @@ struct mv_batch {
     uint8_t *d_mat = nullptr;
     CamRec *d_cams = nullptr;
     uint32_t *d_status = nullptr;
+    int4 *d_overlay = nullptr;          // [O][max_overlay_rects]
+    int32_t *d_overlay_count = nullptr; // [O]
+    uint32_t smem_ov_off = 0;
     // host-side readiness tracking (per env)
     std::vector<uint8_t> has_grid, has_palette;
     int missing_grid = 0, missing_palette = 0;
@@ -100,6 +103,10 @@ int launch_render(mv_batch *b, uint8_t *d_rgb, float *d_depth, int obs_begin, in
     p.sky_rgbx = b->sky_rgbx;
     p.miss_depth = b->desc.miss_depth;
     p.smem_mask_off = b->smem_mask_off; p.smem_rel_off = b->smem_rel_off; p.smem_misc_off = b->smem_misc_off;
+    p.smem_ov_off = b->smem_ov_off;
+    p.overlay = b->d_overlay;
+    p.overlay_count = b->d_overlay_count;
+    p.max_overlay = b->desc.max_overlay_rects;
     render_kernel<kRenderThreads><<<obs_count, kRenderThreads, b->smem_bytes, s>>>(p);
     b->launches++;
     MV_CUDA(b, cudaGetLastError());
@@ -180,7 +187,7 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
         d.max_boxes < 0 || d.max_boxes > 256 || d.width < 8 || d.width > 4096 || (d.width % 8) != 0 ||
         d.height < 4 || d.height > 4096 || (d.height % 4) != 0 || d.palette_size < 1 || d.palette_size > 256 ||
         !(d.hfov_rad > 0.0f) || !(d.hfov_rad < 3.14159f) || !(d.ambient >= 0.0f) || !(d.ambient <= 1.0f) ||
-        !std::isfinite(d.miss_depth) || d.device < 0)
+        !std::isfinite(d.miss_depth) || d.device < 0 || d.max_overlay_rects < 0 || d.max_overlay_rects > 16)
         return MV_ERR_INVALID_ARG;
     const double ln = (double)d.light_dir[0] * d.light_dir[0] + (double)d.light_dir[1] * d.light_dir[1] +
                       (double)d.light_dir[2] * d.light_dir[2];
@@ -210,7 +217,8 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
     b->smem_mask_off = round_up(L.block_bytes, 16);
     b->smem_rel_off = b->smem_mask_off + round_up((uint32_t)(b->tiles_x * b->tiles_y * b->mask_words * 4), 16);
     b->smem_misc_off = b->smem_rel_off + (uint32_t)(d.max_boxes > 0 ? d.max_boxes : 1) * 32;
-    b->smem_bytes = b->smem_misc_off + 16;
+    b->smem_ov_off = b->smem_misc_off + 16;
+    b->smem_bytes = b->smem_ov_off + (uint32_t)(d.max_overlay_rects > 0 ? d.max_overlay_rects : 1) * 32;
 
     // kr = tan(hfov/2)/W, ku = (tan(hfov/2)*H/W)/H in double (scalar set-up for the camera kernel)
     const double tx = std::tan((double)d.hfov_rad / 2.0);
@@ -237,6 +245,10 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
               cudaMalloc(&b->d_mat, (size_t)d.num_envs * b->nvox) == cudaSuccess &&
               cudaMalloc(&b->d_cams, (size_t)b->num_obs * sizeof(CamRec)) == cudaSuccess &&
               cudaMalloc(&b->d_status, 16) == cudaSuccess;
+    if (ok && d.max_overlay_rects > 0)
+        ok = cudaMalloc(&b->d_overlay, (size_t)b->num_obs * d.max_overlay_rects * 16) == cudaSuccess &&
+             cudaMalloc(&b->d_overlay_count, (size_t)b->num_obs * 4) == cudaSuccess &&
+             cudaMemset(b->d_overlay_count, 0, (size_t)b->num_obs * 4) == cudaSuccess;
     if (ok) ok = cudaMemset(b->d_env_blocks, 0, blocks_bytes) == cudaSuccess &&
                  cudaMemset(b->d_status, 0, 16) == cudaSuccess;
     if (!ok) {
@@ -297,6 +309,43 @@ int mv_set_cameras(mv_batch *b, const mv_camera *d_cams, void *cuda_stream) {
     DeviceGuard g(b->desc.device);
     if (!g.ok) return MV_ERR_CUDA;
     return launch_cameras(b, d_cams, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int mv_set_overlays(mv_batch *b, const mv_overlay_rect *d_rects, const int32_t *d_count, void *cuda_stream) {
+    if (!b || (d_rects && !d_count)) return MV_ERR_INVALID_ARG;
+    const int m = b->desc.max_overlay_rects;
+    if (m == 0) return d_rects ? MV_ERR_INVALID_ARG : MV_OK;
+    if (d_rects && !aligned16(d_rects)) return MV_ERR_INVALID_ARG;
+    DeviceGuard g(b->desc.device);
+    if (!g.ok) return MV_ERR_CUDA;
+    const int n = b->num_obs * (m + 1);
+    copy_overlays_kernel<<<(n + 255) / 256, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        reinterpret_cast<const int4 *>(d_rects), d_count, b->d_overlay, b->d_overlay_count, b->num_obs, m);
+    b->launches++;
+    MV_CUDA(b, cudaGetLastError());
+    return MV_OK;
+}
+
+int mv_move_agents(mv_batch *b, mv_camera *d_cams_inout, const mv_agent_move *d_moves, const mv_body_shape *shape,
+                   void *cuda_stream) {
+    if (!b || !d_cams_inout || !d_moves || !aligned16(d_moves)) return MV_ERR_INVALID_ARG;
+    mv_body_shape sh = {0.25f, 0.75f, 0.25f, 1.0f};
+    if (shape) sh = *shape;
+    if (!(sh.half_width >= 0.0f) || !(sh.below_eye >= 0.0f) || !(sh.above_eye >= 0.0f) || !(sh.max_pitch >= 0.0f) ||
+        !(sh.half_width < 16.0f) || !(sh.below_eye < 16.0f) || !(sh.above_eye < 16.0f))
+        return MV_ERR_INVALID_ARG;
+    if (b->missing_grid > 0) return MV_ERR_NOT_READY;
+    DeviceGuard g(b->desc.device);
+    if (!g.ok) return MV_ERR_CUDA;
+    const int n = b->num_obs;
+    move_agents_kernel<<<(n + 127) / 128, 128, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        reinterpret_cast<int32_t *>(d_cams_inout), reinterpret_cast<const float4 *>(d_moves), b->d_cams,
+        b->d_env_blocks, b->lay, n, b->desc.agents_per_env, b->desc.grid_x, b->desc.grid_y, b->desc.grid_z,
+        b->desc.max_boxes, sh.half_width, sh.below_eye, sh.above_eye, sh.max_pitch, b->kr, b->ku, b->d_status);
+    b->launches++;
+    MV_CUDA(b, cudaGetLastError());
+    b->has_cams = true;
+    return MV_OK;
 }
 
 int mv_render_batch(mv_batch *b, uint8_t *d_rgb, float *d_depth, void *cuda_stream) {
@@ -414,6 +463,7 @@ int mv_destroy(mv_batch *b) {
         if (g.ok) {
             if (cudaDeviceSynchronize() != cudaSuccess) rc = MV_ERR_CUDA;
             cudaFree(b->d_env_blocks); cudaFree(b->d_mat); cudaFree(b->d_cams); cudaFree(b->d_status);
+            cudaFree(b->d_overlay); cudaFree(b->d_overlay_count);
             cudaFree(b->d_rgb); cudaFree(b->d_depth); cudaFree(b->d_cam_in); cudaFree(b->d_box_in);
             cudaFree(b->d_count_in);
             if (b->copy_stream) cudaStreamDestroy(b->copy_stream);

@@ -51,6 +51,10 @@ struct RenderParams {
     uint32_t sky_rgbx;
     float miss_depth;
     uint32_t smem_mask_off, smem_rel_off, smem_misc_off;   // offsets after the env block
+    uint32_t smem_ov_off;              // overlay rectangles of the observation
+    const int4 *overlay;               // [O][max_overlay] 16-byte records, or null
+    const int32_t *overlay_count;      // [O]
+    int max_overlay;
 };
 
 }  // namespace mv

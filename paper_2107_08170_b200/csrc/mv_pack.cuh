@@ -137,16 +137,11 @@ __global__ void copy_boxes_kernel(const uint4 *__restrict__ boxes, const int32_t
 // Camera -> ray basis, evaluated in double and rounded to float:
 // F = (cp*sy, sp, cp*cy), R = (cy, 0, -sy), U = (-sp*sy, cp, -sp*cy); Rs = R*kr, Us = U*ku
 // with kr = tan(hfov/2)/W and ku = (tan(hfov/2)*H/W)/H computed on the host in double.
-__global__ void camera_kernel(const int32_t *__restrict__ cams, CamRec *__restrict__ out, int num_obs,
-                              double kr, double ku, uint32_t *status)
+__device__ __forceinline__ void write_camrec(CamRec *out, float px, float py, float pz, float yaw, float pitch,
+                                             int self_box, double kr, double ku, uint32_t *status)
 {
-    const int o = blockIdx.x * blockDim.x + threadIdx.x;
-    if (o >= num_obs) return;
-    const int32_t *c = cams + (size_t)o * 6;
-    const float px = __int_as_float(c[0]), py = __int_as_float(c[1]), pz = __int_as_float(c[2]);
-    const float yaw = __int_as_float(c[3]), pitch = __int_as_float(c[4]);
     CamRec r;
-    r.self_box = c[5];
+    r.self_box = self_box;
     r.pad[0] = r.pad[1] = 0;
     const bool ok = isfinite(px) && isfinite(py) && isfinite(pz) && isfinite(yaw) && isfinite(pitch);
     r.flags = ok ? 0u : kFlagBadCamera;
@@ -158,8 +153,96 @@ __global__ void camera_kernel(const int32_t *__restrict__ cams, CamRec *__restri
     r.Rs[0] = (float)__dmul_rn(cy, kr); r.Rs[1] = (float)__dmul_rn(0.0, kr); r.Rs[2] = (float)__dmul_rn(-sy, kr);
     r.Us[0] = (float)__dmul_rn(__dmul_rn(-sp, sy), ku); r.Us[1] = (float)__dmul_rn(cp, ku);
     r.Us[2] = (float)__dmul_rn(__dmul_rn(-sp, cy), ku);
-    out[o] = r;
+    *out = r;
     if (!ok) atomicOr(status, kFlagBadCamera);
+}
+
+__global__ void camera_kernel(const int32_t *__restrict__ cams, CamRec *__restrict__ out, int num_obs,
+                              double kr, double ku, uint32_t *status)
+{
+    const int o = blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= num_obs) return;
+    const int32_t *c = cams + (size_t)o * 6;
+    write_camrec(out + o, __int_as_float(c[0]), __int_as_float(c[1]), __int_as_float(c[2]),
+                 __int_as_float(c[3]), __int_as_float(c[4]), c[5], kr, ku, status);
+}
+
+// True iff the body box around (x, y, z) lies inside the grid and touches no filled voxel
+// (cells floor(lo)..floor(hi) on every axis, ends included).
+__device__ __forceinline__ bool body_free(const uint32_t *occ, int gx, int gy, int gz, float x, float y, float z,
+                                          float hw, float below, float above)
+{
+    const float lx = __fsub_rn(x, hw), hx = __fadd_rn(x, hw);
+    const float ly = __fsub_rn(y, below), hy = __fadd_rn(y, above);
+    const float lz = __fsub_rn(z, hw), hz = __fadd_rn(z, hw);
+    if (!(lx >= 0.0f) || !(hx < (float)gx) || !(ly >= 0.0f) || !(hy < (float)gy) || !(lz >= 0.0f) ||
+        !(hz < (float)gz))
+        return false;
+    const int i0 = (int)floorf(lx), i1 = (int)floorf(hx), j0 = (int)floorf(ly), j1 = (int)floorf(hy);
+    const int k0 = (int)floorf(lz), k1 = (int)floorf(hz);
+    for (int j = j0; j <= j1; ++j)
+        for (int k = k0; k <= k1; ++k)
+            for (int i = i0; i <= i1; ++i) {
+                const int v = i + gx * (k + gz * j);
+                if ((occ[v >> 5] >> (v & 31)) & 1u) return false;
+            }
+    return true;
+}
+
+// Agent motion with voxel collision; one thread per agent.  Updates the caller's camera array,
+// the ray-basis table and the agent's own body box inside its env block.
+__global__ void move_agents_kernel(int32_t *__restrict__ cams, const float4 *__restrict__ moves,
+                                   CamRec *__restrict__ recs, unsigned char *__restrict__ env_blocks,
+                                   EnvLayout lay, int num_obs, int agents, int gx, int gy, int gz, int max_boxes,
+                                   float hw, float below, float above, float max_pitch, double kr, double ku,
+                                   uint32_t *status)
+{
+    const int o = blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= num_obs) return;
+    int32_t *c = cams + (size_t)o * 6;
+    const float x = __int_as_float(c[0]), y = __int_as_float(c[1]), z = __int_as_float(c[2]);
+    const float4 mv = moves[o];
+    const float yaw = __fadd_rn(__int_as_float(c[3]), mv.z);
+    float pitch = __fadd_rn(__int_as_float(c[4]), mv.w);
+    pitch = pitch > max_pitch ? max_pitch : pitch;
+    pitch = pitch < -max_pitch ? -max_pitch : pitch;
+    double sy, cy;
+    sincos((double)yaw, &sy, &cy);
+    const double sxd = __dadd_rn(__dmul_rn((double)mv.x, sy), __dmul_rn((double)mv.y, cy));
+    const double szd = __dsub_rn(__dmul_rn((double)mv.x, cy), __dmul_rn((double)mv.y, sy));
+    const float x_try = (float)__dadd_rn((double)x, sxd);
+    const float z_try = (float)__dadd_rn((double)z, szd);
+    unsigned char *blk = env_blocks + (size_t)(o / agents) * lay.stride;
+    const uint32_t *occ = reinterpret_cast<const uint32_t *>(blk);
+    float nx = x, nz = z;
+    if (body_free(occ, gx, gy, gz, x_try, y, nz, hw, below, above)) nx = x_try;
+    if (body_free(occ, gx, gy, gz, nx, y, z_try, hw, below, above)) nz = z_try;
+    c[0] = __float_as_int(nx); c[2] = __float_as_int(nz);
+    c[3] = __float_as_int(yaw); c[4] = __float_as_int(pitch);
+    const int self_box = c[5];
+    write_camrec(recs + o, nx, y, nz, yaw, pitch, self_box, kr, ku, status);
+    const int count = *reinterpret_cast<const int *>(blk + lay.count_off);
+    if (self_box >= 0 && self_box < min(count, max_boxes)) {
+        float *b = reinterpret_cast<float *>(blk + lay.box_off) + 8 * self_box;
+        b[0] = __fsub_rn(nx, hw); b[1] = __fsub_rn(y, below); b[2] = __fsub_rn(nz, hw);
+        b[3] = __fadd_rn(nx, hw); b[4] = __fadd_rn(y, above); b[5] = __fadd_rn(nz, hw);
+    }
+}
+
+// GUI rectangles into the library's table; counts clamped to 0..max_rects.
+__global__ void copy_overlays_kernel(const int4 *__restrict__ rects, const int32_t *__restrict__ counts,
+                                     int4 *__restrict__ out_rects, int32_t *__restrict__ out_counts, int num_obs,
+                                     int max_rects)
+{
+    const int gid = blockIdx.x * blockDim.x + threadIdx.x;
+    if (gid >= num_obs * (max_rects + 1)) return;
+    const int o = gid / (max_rects + 1), r = gid - o * (max_rects + 1);
+    if (r == max_rects) {
+        const int n = rects ? counts[o] : 0;
+        out_counts[o] = n < 0 ? 0 : (n > max_rects ? max_rects : n);
+    } else if (rects) {
+        out_rects[(size_t)o * max_rects + r] = rects[(size_t)o * max_rects + r];
+    }
 }
 
 }  // namespace mv

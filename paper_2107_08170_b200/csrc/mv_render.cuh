@@ -101,6 +101,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     uint32_t *s_mask = reinterpret_cast<uint32_t *>(smem + p.smem_mask_off);
     float4 *s_rel = reinterpret_cast<float4 *>(smem + p.smem_rel_off);
     uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + p.smem_misc_off);
+    int4 *s_ov = reinterpret_cast<int4 *>(smem + p.smem_ov_off);
 
     // ---- camera record (64 bytes, same for the whole CTA)
     const float4 *cq = reinterpret_cast<const float4 *>(p.cams + obs);
@@ -131,6 +132,14 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     const int ntiles = p.tiles_x * p.tiles_y;
     const int mw = p.mask_words;
     for (int i = tid; i < ntiles * mw; i += NT) s_mask[i] = 0u;
+    // GUI rectangles of this observation (unpacked to x0,y0,x1,y1 / colour in two slots)
+    const int ov_count = p.overlay ? min(max(__ldg(p.overlay_count + obs), 0), p.max_overlay) : 0;
+    if (tid < ov_count) {
+        const int4 q = __ldg(p.overlay + (size_t)obs * p.max_overlay + tid);
+        s_ov[2 * tid] = make_int4((int)(short)(q.x & 0xffff), (int)(short)(q.x >> 16),
+                                  (int)(short)(q.y & 0xffff), (int)(short)(q.y >> 16));
+        s_ov[2 * tid + 1] = make_int4(q.z & 0xffffff, 0, 0, 0);
+    }
 
     if (!mbar_wait_bounded(s_bar, 0, kWaitPolls)) {
         if (tid == 0) atomicOr(p.status, kFlagTimeout);
@@ -388,6 +397,15 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             const int face = axis < 0 ? kFaceInside : 2 * axis + (ds > 0.0f ? 0 : 1);
             rgbx = s_lut[face * P_ + m];
             depth = t_hit + 0.0f;
+        }
+
+        // ---- GUI overlay: rectangles in list order, later ones on top; depth is left alone
+        if (ov_count > 0) {
+            const int px = txi * 8 + (lane & 7), py = tyi * 4 + (lane >> 3);
+            for (int r = 0; r < ov_count; ++r) {
+                const int4 q = s_ov[2 * r];
+                if (px >= q.x && px < q.z && py >= q.y && py < q.w) rgbx = (uint32_t)s_ov[2 * r + 1].x;
+            }
         }
 
         // ---- store: depth rows are 32-byte segments; RGB rows are 24 bytes = 6 packed words

@@ -27,7 +27,7 @@ def test_header_symbols_are_exported(mvlib):
 
 
 def test_struct_sizes_match_header(mvlib):
-    assert C.sizeof(mvlib.BatchDesc) == 68
+    assert C.sizeof(mvlib.BatchDesc) == 72
 
 
 def test_status_strings(mvlib):

@@ -1,0 +1,133 @@
+"""GUI overlay and agent motion on the GPU (through the C ABI) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2107_08170_b200 import scenes
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _random_rects(oracle, num_obs, max_rects, W, H, seed):
+    rng = np.random.default_rng(seed)
+    rects = np.zeros((num_obs, max_rects), oracle.RECT_DTYPE)
+    count = rng.integers(0, max_rects + 2, size=num_obs).astype(np.int32)       # some beyond the limit
+    for o in range(num_obs):
+        for r in range(max_rects):
+            x0, y0 = int(rng.integers(-8, W)), int(rng.integers(-4, H))
+            rects[o, r] = (x0, y0, x0 + int(rng.integers(0, W // 2)), y0 + int(rng.integers(0, H // 3)),
+                           tuple(int(v) for v in rng.integers(0, 256, 3)), 0, 0)
+        rects[o, 0] = (0, 0, int(rng.integers(0, W + 1)), 2, (250, 240, 30), 0, 0)   # a time-left bar
+    return rects, count
+
+
+def test_overlay_matches_oracle_and_leaves_depth_alone(oracle):
+    from paper_2107_08170_b200 import binding as B
+    from gpu_util import upload_scene, scene_to_numpy
+    cfg = scenes.config("rooms_boxes", num_envs=3)
+    sc = scenes.make_scene(cfg)
+    M = 4
+    batch = B.Batch(B.desc_from_config(cfg, max_overlay_rects=M))
+    upload_scene(batch, sc)
+    batch.set_cameras(sc["cams"].cuda())
+    rgb0, depth0 = batch.alloc_outputs()
+    batch.render_batch(rgb0, depth0)                                          # no overlay yet
+    rects, count = _random_rects(oracle, cfg.num_obs, M, cfg.width, cfg.height, 5)
+    d_rects = torch.from_numpy(rects.view(np.int32).reshape(cfg.num_obs, M, 4)).cuda()
+    batch.set_overlays(d_rects, torch.from_numpy(count).cuda())
+    rgb1, depth1 = batch.alloc_outputs()
+    batch.render_batch(rgb1, depth1)
+    assert torch.equal(depth0, depth1)
+    base = rgb0.cpu().numpy()
+    got = rgb1.cpu().numpy()
+    painted = 0
+    for o in range(cfg.num_obs):
+        want = oracle.overlay(base[o].copy(), rects[o], min(max(int(count[o]), 0), M))
+        assert (got[o] == want).all(), o                                      # integer work: bit-exact
+        painted += int((want != base[o]).any(axis=-1).sum())
+    assert painted > 1000
+    # the 3D part under the overlay is the ordinary render: check it against the oracle too
+    st = parity.compare_scene(oracle, cfg, scene_to_numpy(sc), range(cfg.num_obs), base, depth0.cpu().numpy())
+    parity.assert_parity(st, "overlay base")
+    batch.set_overlays(None, None)
+    rgb2, depth2 = batch.alloc_outputs()
+    batch.render_batch(rgb2, depth2)
+    assert torch.equal(rgb2, rgb0)
+    batch.destroy()
+
+
+def test_move_agents_matches_oracle_then_renders(oracle):
+    from paper_2107_08170_b200 import binding as B
+    from gpu_util import upload_scene, scene_to_numpy
+    cfg = scenes.config("rooms_boxes", num_envs=6)
+    sc = scenes.make_scene(cfg)
+    scn = scene_to_numpy(sc)
+    batch = B.Batch(B.desc_from_config(cfg))
+    upload_scene(batch, sc)
+    d_cams = sc["cams"].cuda().contiguous()
+    cams = scn["cams"].copy()
+    boxes = scn["boxes"].copy()
+    rng = np.random.default_rng(1)
+    shape = (0.25, 0.75, 0.25)
+    mismatched = blocked = 0
+    for step in range(12):
+        moves = np.stack([rng.uniform(-0.45, 0.45, cfg.num_obs), rng.uniform(-0.2, 0.2, cfg.num_obs),
+                          rng.normal(0, 0.3, cfg.num_obs), rng.normal(0, 0.1, cfg.num_obs)], 1).astype(np.float32)
+        batch.move_agents(d_cams, torch.from_numpy(moves).cuda())
+        for o in range(cfg.num_obs):
+            e = o // cfg.agents
+            f = cams[o, :5].view(np.float32)
+            new, kept = oracle.move_agent(scn["grid"][e], f, moves[o], shape, 1.0)
+            blocked += kept != 3
+            cams[o, :5] = new.view(np.int32)
+            sb = cams[o, 5]
+            lo = np.float32(new[:3]) - np.float32([0.25, 0.75, 0.25])
+            hi = np.float32(new[:3]) + np.float32([0.25, 0.25, 0.25])
+            boxes[e, sb, :3] = lo.astype(np.float32).view(np.int32)
+            boxes[e, sb, 3:6] = hi.astype(np.float32).view(np.int32)
+        g = d_cams.cpu().numpy()
+        mismatched += int((g != cams).any(axis=1).sum())
+        cams = g.copy()                          # keep both sides on the same state for the next step
+        for o in range(cfg.num_obs):             # and the boxes the GPU now holds for those agents
+            e = o // cfg.agents
+            f = cams[o, :5].view(np.float32)
+            boxes[e, cams[o, 5], :3] = (f[:3] - np.float32([0.25, 0.75, 0.25])).view(np.int32)
+            boxes[e, cams[o, 5], 3:6] = (f[:3] + np.float32([0.25, 0.25, 0.25])).view(np.int32)
+    assert blocked > 10
+    # double sin/cos differ by an ulp between libm and CUDA at most in rare roundings
+    assert mismatched <= 1, mismatched
+    rgb, depth = batch.alloc_outputs()
+    batch.render_batch(rgb, depth)               # no mv_set_cameras: the move rebuilt the ray bases
+    scn2 = dict(scn, cams=cams, boxes=boxes)
+    st = parity.compare_scene(oracle, cfg, scn2, range(cfg.num_obs), rgb.cpu().numpy(), depth.cpu().numpy())
+    parity.assert_parity(st, "after moves")
+    assert batch.query_status() == 0
+    batch.destroy()
+
+
+def test_move_agents_headline_scale_properties(oracle):
+    """At the headline size: agents never end inside a voxel; yaw/pitch follow the commands."""
+    from paper_2107_08170_b200 import workload
+    cfg = scenes.config("headline", num_envs=2048)
+    batch, d_cams, kept = workload.build_batch(cfg, 0, keep_envs=[0, 1000, 2047])
+    g = torch.Generator(device="cuda").manual_seed(0)
+    # stand every agent with its feet on its surface (eye 0.75 above the cell floor)
+    yf = d_cams[:, 1].contiguous().view(torch.float32)
+    d_cams[:, 1] = (yf.floor() + 0.75).view(torch.int32)
+    for e in kept:
+        kept[e]["cams"][0, 1] = d_cams[e, 1].item()
+    before = d_cams.clone()
+    moves = (torch.rand(cfg.num_obs, 4, device="cuda", generator=g) - 0.5) * torch.tensor([1.0, 0.5, 0.6, 0.2], device="cuda")
+    batch.move_agents(d_cams, moves.contiguous())
+    after = d_cams.cpu().numpy()
+    for e in kept:
+        f0 = kept[e]["cams"][0, :5].view(np.float32)
+        new, _ = oracle.move_agent(kept[e]["grid"], f0, moves[e].cpu().numpy(), (0.25, 0.75, 0.25), 1.0)
+        assert (after[e, :5].view(np.float32) == new).all()
+    fa = np.ascontiguousarray(after[:, :5]).view(np.float32)
+    fb = np.ascontiguousarray(before.cpu().numpy()[:, :5]).view(np.float32)
+    assert np.allclose(fa[:, 3], fb[:, 3] + moves[:, 2].cpu().numpy(), atol=1e-6)
+    assert (np.abs(fa[:, 4]) <= 1.0).all() and (fa[:, 1] == fb[:, 1]).all()
+    assert ((fa[:, 0] != fb[:, 0]) | (fa[:, 2] != fb[:, 2])).mean() > 0.2
+    batch.destroy()
