@@ -132,13 +132,27 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     const int ntiles = p.tiles_x * p.tiles_y;
     const int mw = p.mask_words;
     for (int i = tid; i < ntiles * mw; i += NT) s_mask[i] = 0u;
-    // GUI rectangles of this observation (unpacked to x0,y0,x1,y1 / colour in two slots)
+    // GUI rectangles of this observation (unpacked to x0,y0,x1,y1 / colour in two slots) and one
+    // bit per tile that any rectangle touches, so untouched tiles pay a single bit test
     const int ov_count = p.overlay ? min(max(__ldg(p.overlay_count + obs), 0), p.max_overlay) : 0;
-    if (tid < ov_count) {
-        const int4 q = __ldg(p.overlay + (size_t)obs * p.max_overlay + tid);
-        s_ov[2 * tid] = make_int4((int)(short)(q.x & 0xffff), (int)(short)(q.x >> 16),
-                                  (int)(short)(q.y & 0xffff), (int)(short)(q.y >> 16));
-        s_ov[2 * tid + 1] = make_int4(q.z & 0xffffff, 0, 0, 0);
+    uint32_t *s_ovtile = reinterpret_cast<uint32_t *>(s_ov + 2 * max(p.max_overlay, 1));
+    if (ov_count > 0) {
+        for (int i = tid; i < (ntiles + 31) / 32; i += NT) s_ovtile[i] = 0u;
+        __syncthreads();
+        if (tid < ov_count) {
+            const int4 q = __ldg(p.overlay + (size_t)obs * p.max_overlay + tid);
+            const int x0 = (int)(short)(q.x & 0xffff), y0 = (int)(short)(q.x >> 16);
+            const int x1 = (int)(short)(q.y & 0xffff), y1 = (int)(short)(q.y >> 16);
+            s_ov[2 * tid] = make_int4(x0, y0, x1, y1);
+            s_ov[2 * tid + 1] = make_int4(q.z & 0xffffff, 0, 0, 0);
+            const int cx0 = max(x0, 0), cy0 = max(y0, 0), cx1 = min(x1, W), cy1 = min(y1, H);
+            if (cx0 < cx1 && cy0 < cy1)
+                for (int ty = cy0 >> 2; ty <= ((cy1 - 1) >> 2); ++ty)
+                    for (int tx = cx0 >> 3; tx <= ((cx1 - 1) >> 3); ++tx) {
+                        const int t = ty * p.tiles_x + tx;
+                        atomicOr(&s_ovtile[t >> 5], 1u << (t & 31));
+                    }
+        }
     }
 
     if (!mbar_wait_bounded(s_bar, 0, kWaitPolls)) {
@@ -400,7 +414,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         }
 
         // ---- GUI overlay: rectangles in list order, later ones on top; depth is left alone
-        if (ov_count > 0) {
+        if (ov_count > 0 && ((s_ovtile[tile >> 5] >> (tile & 31)) & 1u)) {
             const int px = txi * 8 + (lane & 7), py = tyi * 4 + (lane >> 3);
             for (int r = 0; r < ov_count; ++r) {
                 const int4 q = s_ov[2 * r];
