@@ -335,3 +335,62 @@ int mvo_move_agent(const uint8_t *grid, int gx, int gy, int gz, float cam[5], co
     cam[0] = x; cam[2] = z; cam[3] = yaw; cam[4] = pitch;
     return kept;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Greedy merging of voxels into boxes (paper Section 3.3: adjacent voxels are merged into a small
+ * number of enclosing parallelepipeds by a greedy O(n) pass at the start of an episode).  The
+ * paper does not spell the pass out; the reading used here is the usual greedy sweep: visit
+ * voxels in index order (x fastest, then z, then y); at the first filled voxel not yet covered,
+ * grow a box along +x while the material is the same and the cells are uncovered, then along +z
+ * while the whole x-run qualifies, then along +y while the whole x-z slab qualifies; emit it and
+ * mark it covered.  Materials are compared after clamping to the palette.
+ * boxes_out: [max_out] records {lo x,y,z, hi x,y,z as float, material, 0}; returns the number of
+ * boxes the pass produces (only the first max_out are written). */
+int mvo_merge_voxels(const uint8_t *grid, int gx, int gy, int gz, int palette_size, mvo_box *boxes_out,
+                     int max_out)
+{
+    size_t n = (size_t)gx * gy * gz;
+    uint8_t *mat = (uint8_t *)malloc(n ? n : 1), *cov = (uint8_t *)calloc(n ? n : 1, 1);
+    if (!mat || !cov) { free(mat); free(cov); return -2; }
+    for (size_t v = 0; v < n; ++v) mat[v] = grid[v] >= palette_size ? (uint8_t)(palette_size - 1) : grid[v];
+#define CELL(i, j, k) (((size_t)(j) * gz + (k)) * gx + (i))
+#define OPEN(i, j, k, m) (grid[CELL(i, j, k)] != 0 && !cov[CELL(i, j, k)] && mat[CELL(i, j, k)] == (m))
+    int count = 0;
+    for (int j = 0; j < gy; ++j)
+        for (int k = 0; k < gz; ++k)
+            for (int i = 0; i < gx; ++i) {
+                if (grid[CELL(i, j, k)] == 0 || cov[CELL(i, j, k)]) continue;
+                int m = mat[CELL(i, j, k)];
+                int w = 1, d = 1, h = 1;
+                while (i + w < gx && OPEN(i + w, j, k, m)) ++w;
+                for (;;) {
+                    if (k + d >= gz) break;
+                    int ok = 1;
+                    for (int a = 0; a < w && ok; ++a) ok = OPEN(i + a, j, k + d, m);
+                    if (!ok) break;
+                    ++d;
+                }
+                for (;;) {
+                    if (j + h >= gy) break;
+                    int ok = 1;
+                    for (int b = 0; b < d && ok; ++b)
+                        for (int a = 0; a < w && ok; ++a) ok = OPEN(i + a, j + h, k + b, m);
+                    if (!ok) break;
+                    ++h;
+                }
+                for (int c = 0; c < h; ++c)
+                    for (int b = 0; b < d; ++b)
+                        for (int a = 0; a < w; ++a) cov[CELL(i + a, j + c, k + b)] = 1;
+                if (count < max_out) {
+                    mvo_box *o = &boxes_out[count];
+                    o->lo[0] = (float)i; o->lo[1] = (float)j; o->lo[2] = (float)k;
+                    o->hi[0] = (float)(i + w); o->hi[1] = (float)(j + h); o->hi[2] = (float)(k + d);
+                    o->material = (uint32_t)m; o->pad = 0;
+                }
+                ++count;
+            }
+#undef CELL
+#undef OPEN
+    free(mat); free(cov);
+    return count;
+}

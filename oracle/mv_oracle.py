@@ -173,3 +173,18 @@ def move_agent(grid, cam5, move4, shape3=(0.25, 0.75, 0.25), max_pitch=1.0):
     kept = L.mvo_move_agent(_ptr(grid, C.c_uint8), C.c_int(gx), C.c_int(gy), C.c_int(gz), _ptr(cam, C.c_float),
                             _ptr(move, C.c_float), _ptr(shape, C.c_float), C.c_float(float(np.float32(max_pitch))))
     return cam, kept
+
+
+def merge_voxels(grid, palette_size, max_out=4096):
+    """Greedy voxel merging of one env: returns (boxes int32[count][8] in the C ABI's box layout,
+    total count the pass produces)."""
+    grid = np.ascontiguousarray(grid, dtype=np.uint8)
+    gy, gz, gx = grid.shape
+    out = np.zeros((max_out, 8), np.int32)
+    L = lib()
+    L.mvo_merge_voxels.restype = C.c_int
+    n = L.mvo_merge_voxels(_ptr(grid, C.c_uint8), C.c_int(gx), C.c_int(gy), C.c_int(gz), C.c_int(palette_size),
+                           out.ctypes.data_as(C.c_void_p), C.c_int(max_out))
+    if n < 0:
+        raise RuntimeError(f"mvo_merge_voxels failed: {n}")
+    return out[:min(n, max_out)], n

@@ -91,3 +91,59 @@ def test_many_random_moves_never_end_inside_a_voxel(oracle):
             assert (g[lo[1]:hi[1] + 1, lo[2]:hi[2] + 1, lo[0]:hi[0] + 1] == 0).all()
         cam = new
     assert blocked > 0
+
+
+def _paint(boxes, shape):
+    gy, gz, gx = shape
+    g = np.zeros(shape, np.int32)
+    hits = np.zeros(shape, np.int32)
+    for b in boxes:
+        lo = b[:3].view(np.float32).astype(int); hi = b[3:6].view(np.float32).astype(int)
+        g[lo[1]:hi[1], lo[2]:hi[2], lo[0]:hi[0]] = b[6]
+        hits[lo[1]:hi[1], lo[2]:hi[2], lo[0]:hi[0]] += 1
+    return g, hits
+
+
+def test_merge_small_cases(oracle):
+    g = np.zeros((4, 4, 4), np.uint8); g[1:3, 1:3, 1:3] = 2
+    boxes, n = oracle.merge_voxels(g, 4)
+    assert n == 1 and boxes[0, :6].view(np.float32).tolist() == [1, 1, 1, 3, 3, 3] and boxes[0, 6] == 2
+    g[1:3, 1:3, 1] = 3                                   # a slab of another material splits it in two
+    boxes, n = oracle.merge_voxels(g, 4)
+    assert n == 2 and sorted(boxes[:, 6].tolist()) == [2, 3]
+    # L shape in one layer: x-run first, so the long arm along x is one box and the rest another
+    g = np.zeros((4, 4, 4), np.uint8); g[0, 0, 0:3] = 1; g[0, 1:3, 0] = 1
+    boxes, n = oracle.merge_voxels(g, 2)
+    assert n == 2
+    assert boxes[0, :6].view(np.float32).tolist() == [0, 0, 0, 3, 1, 1]
+    assert boxes[1, :6].view(np.float32).tolist() == [0, 0, 1, 1, 1, 3]
+    assert oracle.merge_voxels(np.zeros((4, 4, 4), np.uint8), 2)[1] == 0
+
+
+def test_merge_covers_exactly_and_is_compact(oracle):
+    from paper_2107_08170_b200 import scenes
+    for name, bound in (("rooms", 400), ("headline", 3000), ("tiny", 60)):
+        cfg = scenes.config(name, num_envs=2)
+        sc = scenes.make_scene(cfg)
+        g = sc["grid"][1].numpy()
+        boxes, n = oracle.merge_voxels(g, cfg.palette_size, 8192)
+        assert n == len(boxes) and 0 < n <= bound, (name, n)
+        painted, hits = _paint(boxes, g.shape)
+        assert (painted == g).all()                      # union of the boxes is the grid, materials kept
+        assert hits.max() == 1                           # and the boxes are disjoint
+        assert n < int((g != 0).sum()) / 10
+
+
+def test_merged_boxes_render_like_the_grid(oracle):
+    from paper_2107_08170_b200 import scenes
+    cfg = scenes.config("tiny")
+    sc = scenes.make_scene(cfg)
+    g = sc["grid"][2].numpy()
+    boxes, n = oracle.merge_voxels(g, cfg.palette_size, 256)
+    d_grid = oracle.desc_from_config(cfg)
+    d_box = oracle.desc_from_config(cfg); d_box.max_boxes = n
+    cam = sc["cams"][2].numpy()
+    a = oracle.render_obs(d_grid, g, None, 0, sc["palette"][2].numpy(), cam)
+    b = oracle.render_obs(d_box, np.zeros_like(g), boxes, n, sc["palette"][2].numpy(), cam)
+    same = (a[0] == b[0]).all(axis=-1) & (np.abs(a[1] - b[1]) <= 1e-6 * np.maximum(a[1], 1e-3))
+    assert same.mean() > 0.999
