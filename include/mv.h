@@ -158,6 +158,21 @@ int mv_set_cameras(mv_batch *batch, const mv_camera *d_cams, void *cuda_stream);
  * Errors: INVALID_ARG, NOT_READY (some env has no grid/palette yet, or no cameras), CUDA. */
 int mv_render_batch(mv_batch *batch, uint8_t *d_rgb, float *d_depth, void *cuda_stream);
 
+/* Merge the voxels of envs [env_begin, env_begin+env_count) into boxes (paper Section 3.3: at
+ * the start of an episode adjacent voxels are merged greedily into a small number of enclosing
+ * parallelepipeds).  The render path of this library walks the grid and does not need the
+ * merged form; the boxes are for callers that want the paper's compact geometry (a rasteriser, a
+ * physics broad phase) or want to compare box primitives with grid traversal.  Order and shape are
+ * those of a serial sweep in index order (x fastest, then z, then y) that grows each box along
+ * +x, then +z, then +y over cells of one material.
+ *   d_boxes_out DEVICE mv_box [env_count][max_out]; box b of an env is valid for b < min(count, max_out)
+ *   d_count_out DEVICE int32 [env_count]; the number of boxes the sweep produces (may exceed max_out,
+ *               in which case only the first max_out were written)
+ * The first call allocates a scratch bitmap (256 envs x 1 bit per voxel).
+ * Errors: INVALID_ARG, NOT_READY (an env in the range has no grid), OUT_OF_MEMORY, CUDA. */
+int mv_merge_voxels(mv_batch *batch, int env_begin, int env_count, mv_box *d_boxes_out,
+                    int32_t *d_count_out, int max_out, void *cuda_stream);
+
 /* Set the GUI overlay of every observation (paper Appendix A.2).  The rectangles are painted
  * over the RGB frame in list order (later ones on top) by the render kernel's store stage; depth
  * is not touched.  The overlay stays in force until set again.

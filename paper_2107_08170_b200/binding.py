@@ -16,7 +16,7 @@ _lib = None
 MV_OK = 0
 FLAG_MATERIAL_CLAMPED, FLAG_BOX_COUNT_CLAMPED, FLAG_BAD_CAMERA, FLAG_DEVICE_TIMEOUT = 1, 2, 4, 8
 EXPORTS = ["mv_create_batch", "mv_upload_worlds", "mv_set_cameras", "mv_render_batch", "mv_step_host",
-           "mv_step_host_static", "mv_set_overlays", "mv_move_agents", "mv_query_status", "mv_launch_count", "mv_destroy", "mv_status_string"]
+           "mv_step_host_static", "mv_set_overlays", "mv_move_agents", "mv_merge_voxels", "mv_query_status", "mv_launch_count", "mv_destroy", "mv_status_string"]
 
 
 class BatchDesc(C.Structure):
@@ -51,13 +51,14 @@ def lib() -> C.CDLL:
         L.mv_step_host_static.argtypes = [vp, vp, vp, vp, vp]
         L.mv_set_overlays.argtypes = [vp, vp, vp, vp]
         L.mv_move_agents.argtypes = [vp, vp, vp, vp, vp]
+        L.mv_merge_voxels.argtypes = [vp, i, i, vp, vp, i, vp]
         L.mv_query_status.argtypes = [vp, i, vp]
         L.mv_launch_count.argtypes = [vp]
         L.mv_launch_count.restype = C.c_int64
         L.mv_destroy.argtypes = [vp]
         L.mv_status_string.argtypes = [i]
         L.mv_status_string.restype = C.c_char_p
-        for n in EXPORTS[:9] + ["mv_destroy"]:
+        for n in EXPORTS[:10] + ["mv_destroy"]:
             getattr(L, n).restype = i
         _lib = L
     return _lib
@@ -166,6 +167,15 @@ class Batch:
             sp = C.byref(BodyShape(*shape))
         _check(lib().mv_move_agents(self._h, _dptr(cams, torch.int32), _dptr(moves, torch.float32), sp,
                                     _stream(stream)), "mv_move_agents")
+
+    def merge_voxels(self, env_begin, env_count, max_out, stream=None):
+        """Greedy voxel merge; returns (boxes int32 [env_count][max_out][8], counts int32 [env_count]) on the GPU."""
+        dev = torch.device("cuda", self.desc.device)
+        boxes = torch.zeros(env_count, max_out, 8, dtype=torch.int32, device=dev)
+        counts = torch.zeros(env_count, dtype=torch.int32, device=dev)
+        _check(lib().mv_merge_voxels(self._h, env_begin, env_count, _dptr(boxes), _dptr(counts), max_out,
+                                     _stream(stream)), "mv_merge_voxels")
+        return boxes, counts
 
     def step_host_static(self, cams, rgb, depth, stream=None):
         """The never-allocating host step (fixed 8 MiB device array inside the library): for callers

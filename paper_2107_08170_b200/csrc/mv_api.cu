@@ -20,6 +20,7 @@ namespace {
 #endif
 constexpr int kRenderThreads = MV_NT;
 constexpr int kHostChunks = 8;
+constexpr int kMergeChunk = 256;        // envs merged per launch (bounds the scratch)
 
 inline uint32_t round_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
 
@@ -34,6 +35,7 @@ struct mv_batch {
     uint8_t *d_mat = nullptr;
     CamRec *d_cams = nullptr;
     uint32_t *d_status = nullptr;
+    uint32_t *d_covered = nullptr;      // merge scratch: one bit per voxel for kMergeChunk envs
     int4 *d_overlay = nullptr;          // [O][max_overlay_rects]
     int32_t *d_overlay_count = nullptr; // [O]
     uint32_t smem_ov_off = 0;
@@ -349,6 +351,31 @@ int mv_move_agents(mv_batch *b, mv_camera *d_cams_inout, const mv_agent_move *d_
     return MV_OK;
 }
 
+int mv_merge_voxels(mv_batch *b, int env_begin, int env_count, mv_box *d_boxes_out, int32_t *d_count_out,
+                    int max_out, void *cuda_stream) {
+    if (!b || env_begin < 0 || env_count < 0 || (int64_t)env_begin + env_count > b->desc.num_envs || !d_boxes_out ||
+        !d_count_out || max_out < 1 || !aligned16(d_boxes_out))
+        return MV_ERR_INVALID_ARG;
+    for (int e = env_begin; e < env_begin + env_count; ++e)
+        if (!b->has_grid[e]) return MV_ERR_NOT_READY;
+    if (env_count == 0) return MV_OK;
+    DeviceGuard g(b->desc.device);
+    if (!g.ok) return MV_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t words = b->nvox / 32;
+    if (!b->d_covered) MV_CUDA(b, cudaMalloc(&b->d_covered, (size_t)kMergeChunk * words * 4));
+    for (int e0 = 0; e0 < env_count; e0 += kMergeChunk) {
+        const int n = env_count - e0 < kMergeChunk ? env_count - e0 : kMergeChunk;
+        MV_CUDA(b, cudaMemsetAsync(b->d_covered, 0, (size_t)n * words * 4, s));
+        merge_voxels_kernel<<<(n * 32 + 127) / 128, 128, 0, s>>>(
+            b->d_env_blocks, b->d_mat, b->lay, env_begin + e0, n, b->desc.grid_x, b->desc.grid_y, b->desc.grid_z,
+            b->d_covered, reinterpret_cast<uint4 *>(d_boxes_out + (size_t)e0 * max_out), d_count_out + e0, max_out);
+        b->launches++;
+        MV_CUDA(b, cudaGetLastError());
+    }
+    return MV_OK;
+}
+
 int mv_render_batch(mv_batch *b, uint8_t *d_rgb, float *d_depth, void *cuda_stream) {
     if (!b || !d_rgb || !d_depth || !aligned16(d_rgb) || !aligned16(d_depth)) return MV_ERR_INVALID_ARG;
     if (b->missing_grid > 0 || b->missing_palette > 0 || !b->has_cams) return MV_ERR_NOT_READY;
@@ -464,7 +491,7 @@ int mv_destroy(mv_batch *b) {
         if (g.ok) {
             if (cudaDeviceSynchronize() != cudaSuccess) rc = MV_ERR_CUDA;
             cudaFree(b->d_env_blocks); cudaFree(b->d_mat); cudaFree(b->d_cams); cudaFree(b->d_status);
-            cudaFree(b->d_overlay); cudaFree(b->d_overlay_count);
+            cudaFree(b->d_overlay); cudaFree(b->d_overlay_count); cudaFree(b->d_covered);
             cudaFree(b->d_rgb); cudaFree(b->d_depth); cudaFree(b->d_cam_in); cudaFree(b->d_box_in);
             cudaFree(b->d_count_in);
             if (b->copy_stream) cudaStreamDestroy(b->copy_stream);

@@ -229,6 +229,84 @@ __global__ void move_agents_kernel(int32_t *__restrict__ cams, const float4 *__r
     }
 }
 
+// Greedy merging of an env's voxels into boxes (paper Section 3.3), one warp per env, in the
+// same order as a serial sweep: the warp finds the first filled, uncovered voxel in index order,
+// grows a box along +x, then +z, then +y while every cell of the new row / slab is filled,
+// uncovered and of the same material, emits it and marks it covered.  `covered` is scratch:
+// one bit per voxel per env of this launch, zeroed by the caller; it is read around L1 (ld.cg)
+// because lanes read bits that other lanes set with atomics.
+__global__ void merge_voxels_kernel(const unsigned char *__restrict__ env_blocks, const uint8_t *__restrict__ mat,
+                                    EnvLayout lay, int env_begin, int env_count, int gx, int gy, int gz,
+                                    uint32_t *__restrict__ covered, uint4 *__restrict__ boxes_out,
+                                    int32_t *__restrict__ count_out, int max_out)
+{
+    const int lane = threadIdx.x & 31;
+    const int e = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (e >= env_count) return;
+    const size_t nvox = (size_t)gx * gy * gz;
+    const int nwords = (int)(nvox / 32);
+    const uint32_t *occ = reinterpret_cast<const uint32_t *>(env_blocks + (size_t)(env_begin + e) * lay.stride);
+    const uint8_t *m_env = mat + (size_t)(env_begin + e) * nvox;
+    uint32_t *cov = covered + (size_t)e * nwords;
+    uint4 *out = boxes_out + (size_t)e * max_out * 2;
+    const unsigned full = 0xffffffffu;
+    auto open = [&](int i, int j, int k, int m) -> bool {
+        const int v = i + gx * (k + gz * j);
+        const uint32_t bit = 1u << (v & 31);
+        return (occ[v >> 5] & bit) && !(__ldcg(&cov[v >> 5]) & bit) && m_env[v] == m;
+    };
+    int count = 0;
+    for (int w0 = 0; w0 < nwords; w0 += 32) {
+        // words w0..w0+31: lane owns one; handle every uncovered filled voxel in them, in order
+        // every trip covers at least one voxel of these 1024, so 1024 trips always suffice
+        for (int trip = 0; trip < 1024; ++trip) {
+            const int wi = w0 + lane;
+            const uint32_t mine = wi < nwords ? (occ[wi] & ~__ldcg(&cov[wi])) : 0u;
+            const unsigned has = __ballot_sync(full, mine != 0u);
+            if (!has) break;
+            const int src = __ffs(has) - 1;
+            const uint32_t word = __shfl_sync(full, mine, src);
+            const int v = (w0 + src) * 32 + (__ffs(word) - 1);
+            const int i = v % gx, r = v / gx, k = r % gz, j = r / gz;
+            const int m = m_env[v];
+            int w = 1, d = 1, h = 1;
+            for (;;) {                                           // +x, 32 cells per vote
+                const int a = w + lane;
+                const bool ok = (i + a < gx) && open(i + a, j, k, m);
+                const unsigned bad = ~__ballot_sync(full, ok);
+                if (bad) { w += __ffs(bad) - 1; break; }
+                w += 32;
+            }
+            for (; k + d < gz; ++d) {                            // +z, one row per trip
+                bool ok = true;
+                for (int a = lane; a < w; a += 32) ok = ok && open(i + a, j, k + d, m);
+                if (!__all_sync(full, ok)) break;
+            }
+            for (; j + h < gy; ++h) {                            // +y, one slab per trip
+                bool ok = true;
+                for (int c = lane; c < w * d; c += 32) ok = ok && open(i + c % w, j + h, k + c / w, m);
+                if (!__all_sync(full, ok)) break;
+            }
+            __syncwarp();
+            for (int c = lane; c < w * d * h; c += 32) {         // mark covered
+                const int a = c % w, b = (c / w) % d, cc = c / (w * d);
+                const int vv = (i + a) + gx * ((k + b) + gz * (j + cc));
+                atomicOr(&cov[vv >> 5], 1u << (vv & 31));
+            }
+            __threadfence();                                     // marks visible to the other lanes' reads
+            __syncwarp();
+            if (lane == 0 && count < max_out) {
+                out[2 * count] = make_uint4(__float_as_uint((float)i), __float_as_uint((float)j),
+                                            __float_as_uint((float)k), __float_as_uint((float)(i + w)));
+                out[2 * count + 1] = make_uint4(__float_as_uint((float)(j + h)), __float_as_uint((float)(k + d)),
+                                                (uint32_t)m, 0u);
+            }
+            ++count;
+        }
+    }
+    if (lane == 0) count_out[e] = count;
+}
+
 // GUI rectangles into the library's table; counts clamped to 0..max_rects.
 __global__ void copy_overlays_kernel(const int4 *__restrict__ rects, const int32_t *__restrict__ counts,
                                      int4 *__restrict__ out_rects, int32_t *__restrict__ out_counts, int num_obs,
