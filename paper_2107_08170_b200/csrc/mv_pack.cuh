@@ -53,8 +53,17 @@ __global__ void occupied_bounds_kernel(unsigned char *__restrict__ env_blocks, E
     const uint32_t *occ = reinterpret_cast<const uint32_t *>(blk);
     const int nwords = gx * gy * gz / 32;
     int lo[3] = {gx, gy, gz}, hi[3] = {-1, -1, -1};
+    const bool row_aligned = (gx % 32) == 0;       // then a 32-voxel word lies inside one x-row
     for (int w = threadIdx.x; w < nwords; w += blockDim.x) {
         uint32_t m = occ[w];
+        if (!m) continue;
+        if (row_aligned) {
+            const int v = w * 32, x = v % gx, r = v / gx, z = r % gz, y = r / gz;
+            lo[0] = min(lo[0], x + __ffs(m) - 1); hi[0] = max(hi[0], x + 31 - __clz(m));
+            lo[1] = min(lo[1], y); hi[1] = max(hi[1], y);
+            lo[2] = min(lo[2], z); hi[2] = max(hi[2], z);
+            continue;
+        }
         while (m) {
             const int v = w * 32 + (__ffs(m) - 1);
             m &= m - 1;

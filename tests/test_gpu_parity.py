@@ -304,3 +304,25 @@ def test_not_ready_and_argument_errors():
     batch.render_batch(rgb, depth)
     assert batch.query_status() == 0
     batch.destroy()
+
+
+def test_limits_are_reported_not_faulted():
+    B = _binding()
+    import ctypes as C
+    # occupancy of 1024 x 64 x 1024 voxels is 8 MiB: far beyond shared memory -> UNSUPPORTED, no launch
+    d = B.make_desc(1, 1, (1024, 64, 1024), 0, 64, 36, 16)
+    h = C.c_void_p()
+    assert B.lib().mv_create_batch(C.byref(d), C.byref(h)) == -6 and not h.value
+
+
+def test_odd_grid_sizes_and_occupied_bounds(oracle):
+    rng = np.random.default_rng(2)
+    for gx in (20, 32, 44):
+        grid = ((rng.random((2, 8, 12, gx)) < 0.1) * rng.integers(1, 4, size=(2, 8, 12, gx))).astype(np.uint8)
+        grid[:, 5:] = 0                                  # nothing above y = 5
+        grid[:, :, :, :3] = 0                            # nothing left of x = 3
+        grid[1] = 0                                      # env 1 is empty
+        cams = np.stack([cam_row(gx / 2 + 0.3, 6.5, 6.2, 0.4, -0.5), cam_row(2.2, 3.3, 4.4, 1.0, 0.1)])
+        g_rgb, g_depth, status, st = _render_custom(oracle, grid, _pal(2, 4), cams, 64, 36)
+        parity.assert_parity(st, f"gx={gx}")
+        assert (g_depth[1] == 0).all() and (g_depth[0] > 0).mean() > 0.2
