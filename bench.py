@@ -30,6 +30,9 @@ WORKLOAD = "headline"
 # DRAM bytes (read 1.24 GB + write 1.01 GB) of one render_kernel launch on this full workload, from
 # the one-pass ncu capture summarised in profiles/render_kernel_headline_launch_list.md.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 2.25e9
+# Warp instructions the render kernel executes per 8x4-pixel tile on this workload
+# (smsp__inst_executed.sum / tiles, profiles/render_kernel_headline_2048env_ncu_full.md).
+NCU_WARP_INSTRUCTIONS_PER_TILE = 464
 
 
 def measured_peak():
@@ -296,8 +299,14 @@ def main():
                          "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "algorithmic_bytes_per_launch": alg,
                          "kernel_ms_mean": k_ms, "kernel_ms_min": min(render_ms), "kernel_ms_median": statistics.median(render_ms)},
+            # the resource that actually binds: warp-instruction issue slots (one per scheduler per cycle)
+            "issue_roofline": {"bound": "alu", "unit": "warp-instructions/s",
+                               "achieved": NCU_WARP_INSTRUCTIONS_PER_TILE * (cfg.num_obs * px / 32) / (k_ms * 1e-3),
+                               "peak": 148 * 4 * (clocks.get("sm_mhz") or 1965.0) * 1e6,
+                               "peak_kind": "148 SMs x 4 schedulers x sampled SM clock"},
             "paper_context": "paper: 1.1e6 obs/s whole simulator on one 8x RTX 2080 Ti node (128x72 RGB, no depth)",
         }
+        out["issue_roofline"]["frac"] = out["issue_roofline"]["achieved"] / out["issue_roofline"]["peak"]
         if e2e:
             out["e2e"] = {"value": obs_total / (e2e[0] * 1e-3), "unit": "obs/s", "ms_per_step": e2e[0],
                           "h2d_bytes_per_step": e2e[1], "d2h_bytes_per_step": e2e[2], "steps": e2e[3]}

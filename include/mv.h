@@ -249,6 +249,14 @@ int mv_query_status(mv_batch *batch, int clear, void *cuda_stream);
 /* Number of kernels of this library launched on behalf of `batch` so far (host counter). */
 int64_t mv_launch_count(const mv_batch *batch);
 
+/* Failure-detection test hook (no counterpart in the paper).  The render kernel's only device-side
+ * wait is the bounded wait for the staged env block; with skip_staging != 0 the copy is not issued,
+ * so every CTA's wait runs out after wait_polls polls, the kernel returns without touching the
+ * outputs and MV_FLAG_DEVICE_TIMEOUT is set (mv_query_status then returns MV_ERR_DEVICE_TIMEOUT).
+ * Nothing faults or hangs and the context stays usable.  Defaults: skip_staging 0, wait_polls
+ * 2^18; wait_polls must be in 1..2^24.  Host-only call.  Errors: INVALID_ARG. */
+int mv_debug_staging(mv_batch *batch, int skip_staging, int wait_polls);
+
 /* Free everything mv_create_batch allocated (synchronises the device). NULL is accepted. */
 int mv_destroy(mv_batch *batch);
 

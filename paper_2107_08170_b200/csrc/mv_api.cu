@@ -48,6 +48,8 @@ struct mv_batch {
     uint32_t smem_mask_off = 0, smem_rel_off = 0, smem_misc_off = 0, smem_bytes = 0;
     int tiles_x = 0, tiles_y = 0, mask_words = 0;
     int64_t launches = 0;
+    int wait_polls = 1 << 18;
+    int skip_staging = 0;
     int last_cuda_error = 0;
     // mv_step_host resources (allocated on first use)
     uint8_t *d_rgb = nullptr;
@@ -109,6 +111,8 @@ int launch_render(mv_batch *b, uint8_t *d_rgb, float *d_depth, int obs_begin, in
     p.overlay = b->d_overlay;
     p.overlay_count = b->d_overlay_count;
     p.max_overlay = b->desc.max_overlay_rects;
+    p.wait_polls = b->wait_polls;
+    p.skip_staging = b->skip_staging;
     render_kernel<kRenderThreads><<<obs_count, kRenderThreads, b->smem_bytes, s>>>(p);
     b->launches++;
     MV_CUDA(b, cudaGetLastError());
@@ -482,6 +486,13 @@ int mv_query_status(mv_batch *b, int clear, void *cuda_stream) {
 }
 
 int64_t mv_launch_count(const mv_batch *b) { return b ? b->launches : 0; }
+
+int mv_debug_staging(mv_batch *b, int skip_staging, int wait_polls) {
+    if (!b || wait_polls < 1 || wait_polls > (1 << 24)) return MV_ERR_INVALID_ARG;
+    b->skip_staging = skip_staging ? 1 : 0;
+    b->wait_polls = wait_polls;
+    return MV_OK;
+}
 
 int mv_destroy(mv_batch *b) {
     if (!b) return MV_OK;

@@ -55,6 +55,8 @@ struct RenderParams {
     const int4 *overlay;               // [O][max_overlay] 16-byte records, or null
     const int32_t *overlay_count;      // [O]
     int max_overlay;
+    int wait_polls;                    // bound of the staging wait
+    int skip_staging;                  // test hook: the block copy is not issued, so the wait runs out
 };
 
 }  // namespace mv

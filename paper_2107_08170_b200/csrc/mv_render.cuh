@@ -52,7 +52,6 @@ __device__ __forceinline__ float fast_rcp(float x) {
     asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
     return r;
 }
-constexpr int kWaitPolls = 1 << 18;
 
 // One DDA step (see the loop in render_kernel): operands %6..%8 = dt, %9..%11 = t0, %12..%14 =
 // index strides, %15 = grid-exit time, %17 = last occupancy word, %18 = shared base address.
@@ -125,7 +124,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     // ---- stage the environment block
     if (tid == 0) mbar_init(s_bar, 1);
     __syncthreads();
-    if (tid == 0) {
+    if (tid == 0 && !p.skip_staging) {
         mbar_expect_tx(s_bar, p.lay.block_bytes);
         bulk_load(smem, p.env_blocks + (size_t)env * p.lay.stride, p.lay.block_bytes, s_bar);
     }
@@ -155,9 +154,9 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         }
     }
 
-    if (!mbar_wait_bounded(s_bar, 0, kWaitPolls)) {
+    if (!mbar_wait_bounded(s_bar, 0, p.wait_polls)) {
         if (tid == 0) atomicOr(p.status, kFlagTimeout);
-        mbar_wait_bounded(s_bar, 0, kWaitPolls);   // let the copy in flight land before leaving
+        mbar_wait_bounded(s_bar, 0, p.wait_polls);   // let a copy in flight land before leaving
         return;
     }
     __syncthreads();

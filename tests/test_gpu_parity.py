@@ -326,3 +326,29 @@ def test_odd_grid_sizes_and_occupied_bounds(oracle):
         g_rgb, g_depth, status, st = _render_custom(oracle, grid, _pal(2, 4), cams, 64, 36)
         parity.assert_parity(st, f"gx={gx}")
         assert (g_depth[1] == 0).all() and (g_depth[0] > 0).mean() > 0.2
+
+
+def test_bounded_wait_runs_out_and_reports_a_status():
+    """Failure detection without a fault: the staging copy is withheld, every CTA's bounded wait gives
+    up, the host reads a timeout status, and the same batch renders normally afterwards."""
+    from gpu_util import upload_scene
+    B = _binding()
+    cfg = scenes.config("tiny")
+    sc = scenes.make_scene(cfg)
+    batch = B.Batch(B.desc_from_config(cfg))
+    upload_scene(batch, sc)
+    batch.set_cameras(sc["cams"].cuda())
+    rgb, depth = batch.alloc_outputs()
+    batch.render_batch(rgb, depth)
+    good = rgb.clone()
+    rgb.fill_(9)
+    batch.debug_staging(True, 64)
+    batch.render_batch(rgb, depth)
+    with pytest.raises(B.MvError) as ei:
+        batch.query_status(clear=True)
+    assert ei.value.code == -5
+    assert bool((rgb == 9).all())                       # the kernel left the outputs alone
+    batch.debug_staging(False)
+    batch.render_batch(rgb, depth)
+    assert batch.query_status() == 0 and torch.equal(rgb, good)
+    batch.destroy()
