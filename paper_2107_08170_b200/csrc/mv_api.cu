@@ -20,7 +20,7 @@ namespace {
 #endif
 constexpr int kRenderThreads = MV_NT;
 constexpr int kHostChunks = 8;
-constexpr int kMergeChunk = 256;        // envs merged per launch (bounds the scratch)
+constexpr size_t kMergeScratchBytes = 256u << 20;   // coverage bitmap for the envs of one merge launch
 
 inline uint32_t round_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
 
@@ -35,7 +35,8 @@ struct mv_batch {
     uint8_t *d_mat = nullptr;
     CamRec *d_cams = nullptr;
     uint32_t *d_status = nullptr;
-    uint32_t *d_covered = nullptr;      // merge scratch: one bit per voxel for kMergeChunk envs
+    uint32_t *d_covered = nullptr;      // merge scratch: one bit per voxel for merge_chunk envs
+    int merge_chunk = 0;
     int4 *d_overlay = nullptr;          // [O][max_overlay_rects]
     int32_t *d_overlay_count = nullptr; // [O]
     uint32_t smem_ov_off = 0;
@@ -367,7 +368,13 @@ int mv_merge_voxels(mv_batch *b, int env_begin, int env_count, mv_box *d_boxes_o
     if (!g.ok) return MV_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const size_t words = b->nvox / 32;
-    if (!b->d_covered) MV_CUDA(b, cudaMalloc(&b->d_covered, (size_t)kMergeChunk * words * 4));
+    if (!b->d_covered) {
+        size_t chunk = kMergeScratchBytes / (words * 4);
+        chunk = chunk < 1 ? 1 : (chunk > (size_t)b->desc.num_envs ? (size_t)b->desc.num_envs : chunk);
+        MV_CUDA(b, cudaMalloc(&b->d_covered, chunk * words * 4));
+        b->merge_chunk = (int)chunk;
+    }
+    const int kMergeChunk = b->merge_chunk;
     for (int e0 = 0; e0 < env_count; e0 += kMergeChunk) {
         const int n = env_count - e0 < kMergeChunk ? env_count - e0 : kMergeChunk;
         MV_CUDA(b, cudaMemsetAsync(b->d_covered, 0, (size_t)n * words * 4, s));
