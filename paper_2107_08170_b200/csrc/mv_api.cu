@@ -224,7 +224,7 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
     b->smem_mask_off = round_up(L.block_bytes, 16);
     b->smem_rel_off = b->smem_mask_off + round_up((uint32_t)(b->tiles_x * b->tiles_y * b->mask_words * 4), 16);
     b->smem_misc_off = b->smem_rel_off + (uint32_t)(d.max_boxes > 0 ? d.max_boxes : 1) * 32;
-    b->smem_ov_off = b->smem_misc_off + 16;
+    b->smem_ov_off = b->smem_misc_off + 16 + 6 * 16;   // barrier word, then the 6-entry DDA start table
     b->smem_bytes = b->smem_ov_off + (uint32_t)(d.max_overlay_rects > 0 ? d.max_overlay_rects : 1) * 32 +
                     round_up((uint32_t)((b->tiles_x * b->tiles_y + 31) / 32) * 4, 16);
 

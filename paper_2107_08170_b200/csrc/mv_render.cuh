@@ -101,6 +101,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     float4 *s_rel = reinterpret_cast<float4 *>(smem + p.smem_rel_off);
     uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + p.smem_misc_off);
     int4 *s_ov = reinterpret_cast<int4 *>(smem + p.smem_ov_off);
+    float4 *s_dda = reinterpret_cast<float4 *>(smem + p.smem_misc_off + 16);
 
     // ---- camera record (64 bytes, same for the whole CTA)
     const float4 *cq = reinterpret_cast<const float4 *>(p.cams + obs);
@@ -221,13 +222,20 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     if (cam_in) { cx0 = (int)floorf(Px); cy0 = (int)floorf(Py); cz0 = (int)floorf(Pz); }
     const int vi0 = cx0 + stride_z * cz0 + stride_y * cy0;
     const bool start_filled = cam_in && ((s_occ[vi0 >> 5] >> (vi0 & 31)) & 1u);
-    // distance from the eye to the two faces of its cell, and cells left before the box ends
-    const float fposx = (float)(cx0 + 1) - Px, fnegx = (float)cx0 - Px;
-    const float fposy = (float)(cy0 + 1) - Py, fnegy = (float)cy0 - Py;
-    const float fposz = (float)(cz0 + 1) - Pz, fnegz = (float)cz0 - Pz;
-    const float nposx = (float)(hix - 1 - cx0), nnegx = (float)(cx0 - lox);
-    const float nposy = (float)(hiy - 1 - cy0), nnegy = (float)(cy0 - loy);
-    const float nposz = (float)(hiz - 1 - cz0), nnegz = (float)(cz0 - loz);
+    // DDA start table, entry 2*axis + (direction component negative): x = signed distance from the
+    // eye to the cell face the ray meets first, y = cells left before the box ends that way,
+    // z = voxel-index stride (as int bits).  Looked up per ray instead of recomputed.
+    if (tid < 6) {
+        const int ax = tid >> 1, neg = tid & 1;
+        const int c0 = ax == 0 ? cx0 : (ax == 1 ? cy0 : cz0);
+        const float Pc = ax == 0 ? Px : (ax == 1 ? Py : Pz);
+        const int lo_c = ax == 0 ? lox : (ax == 1 ? loy : loz), hi_c = ax == 0 ? hix : (ax == 1 ? hiy : hiz);
+        const int st = ax == 0 ? 1 : (ax == 1 ? stride_y : stride_z);
+        s_dda[tid] = make_float4(neg ? (float)c0 - Pc : (float)(c0 + 1) - Pc,
+                                 neg ? (float)(c0 - lo_c) : (float)(hi_c - 1 - c0),
+                                 __int_as_float(neg ? -st : st), 0.0f);
+    }
+    __syncthreads();
     const int max_steps = gx + gy + gz + 3;
     const uint8_t *mat_env = p.mat + (size_t)env * nvox;
     const int P_ = p.palette;
@@ -246,10 +254,10 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     const int depth_lane_off = (lane >> 3) * W + (lane & 7);
     const int rgb_lane_off = st_r * W * 3 + st_j * 4;
     int tile_px = (tyi * 4) * W + txi * 8;          // first pixel of the warp's current tile
+    // a = 2px+1-W and b = H-1-2py of the lane's pixel, kept as floats (small integers: exact)
+    float a = (float)(16 * txi + 1 - W) + lane_a, bb = (float)(H - 1 - 8 * tyi) - lane_b;
     for (int tile = warp; tile < ntiles; tile += kWarps) {
         // ---- ray through the pixel centre: d = F + a*Rs + b*Us, a = 2px+1-W, b = H-1-2py
-        const float a = (float)(16 * txi + 1 - W) + lane_a;
-        const float bb = (float)(H - 1 - 8 * tyi) - lane_b;
         float dx = fmaf(bb, Ux, fmaf(a, Rx, Fx));
         float dy = fmaf(bb, Uy, fmaf(a, Ry, Fy));
         float dz = fmaf(bb, Uz, fmaf(a, Rz, Fz));
@@ -261,9 +269,10 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         const float ix = fast_rcp(dx), iy = fast_rcp(dy), iz = fast_rcp(dz);
         const bool ngx = dx < 0.0f, ngy = dy < 0.0f, ngz = dz < 0.0f;
         const float dtx = fabsf(ix), dty = fabsf(iy), dtz = fabsf(iz);
-        const int sx = ngx ? -1 : 1;
-        const int sy = ngy ? -stride_y : stride_y;
-        const int sz = ngz ? -stride_z : stride_z;
+        const float4 qx = s_dda[0 + (__float_as_uint(dx) >> 31)];
+        const float4 qy = s_dda[2 + (__float_as_uint(dy) >> 31)];
+        const float4 qz = s_dda[4 + (__float_as_uint(dz) >> 31)];
+        const int sx = __float_as_int(qx.z), sy = __float_as_int(qy.z), sz = __float_as_int(qz.z);
 
         // ---- grid traversal: crossing times are t0 + k*dt with integer-valued k, so the exit
         // time below is bit-identical to the crossing that would leave the grid
@@ -271,11 +280,10 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         int vi = vi0, axis0 = -1;
         bool vhit = start_filled;
         if (cam_in) {
-            t0x = (ngx ? fnegx : fposx) * ix;
-            t0y = (ngy ? fnegy : fposy) * iy;
-            t0z = (ngz ? fnegz : fposz) * iz;
-            t_exit = fminf(fmaf(ngx ? nnegx : nposx, dtx, t0x),
-                           fminf(fmaf(ngy ? nnegy : nposy, dty, t0y), fmaf(ngz ? nnegz : nposz, dtz, t0z)));
+            t0x = qx.x * ix;
+            t0y = qy.x * iy;
+            t0z = qz.x * iz;
+            t_exit = fminf(fmaf(qx.y, dtx, t0x), fminf(fmaf(qy.y, dty, t0y), fmaf(qz.y, dtz, t0z)));
         } else {
             // eye outside the occupied box: clip the ray to it, start in the entry cell
             const float x1 = ((float)lox - Px) * ix, x2 = ((float)hix - Px) * ix;
@@ -431,7 +439,8 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         }
         txi += kWarps;
         tile_px += 8 * kWarps;
-        while (txi >= p.tiles_x) { txi -= p.tiles_x; ++tyi; tile_px += 3 * W; }
+        a += (float)(16 * kWarps);
+        while (txi >= p.tiles_x) { txi -= p.tiles_x; ++tyi; tile_px += 3 * W; a -= (float)(2 * W); bb -= 8.0f; }
     }
 }
 
