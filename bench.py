@@ -32,7 +32,7 @@ WORKLOAD = "headline"
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 2.25e9
 # Warp instructions the render kernel executes per 8x4-pixel tile on this workload
 # (smsp__inst_executed.sum / tiles, profiles/render_kernel_headline_2048env_ncu_full.md).
-NCU_WARP_INSTRUCTIONS_PER_TILE = 464
+NCU_WARP_INSTRUCTIONS_PER_TILE = 435
 
 
 def measured_peak():
