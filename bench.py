@@ -104,6 +104,16 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["clock sampling unavailable"]}
 
 
+def cpu_model() -> str:
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def cpu_oracle_rate(cfg, kept, max_seconds=25.0, max_obs=8):
     """Observations per second of the oracle, as it stands, on this host's cores."""
     from oracle import mv_oracle
@@ -155,7 +165,8 @@ def run_reference(args, rank):
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": workload_config(cfg, args.gpus),
-        "cpu_baseline": {"value": value, "unit": "obs/s", "cores": cores, "kind": "oracle", "sample": what},
+        "cpu_baseline": {"value": value, "unit": "obs/s", "cores": cores, "kind": "oracle", "cpu_model": cpu_model(),
+                         "sample": what},
         "e2e": {"value": value, "unit": "obs/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
@@ -312,7 +323,7 @@ def main():
                           "h2d_bytes_per_step": e2e[1], "d2h_bytes_per_step": e2e[2], "steps": e2e[3]}
         if not args.no_cpu and kept:
             rate, n, secs, cores = cpu_oracle_rate(cfg, kept)
-            out["cpu_baseline"] = {"value": rate, "unit": "obs/s", "cores": cores, "kind": "oracle",
+            out["cpu_baseline"] = {"value": rate, "unit": "obs/s", "cores": cores, "kind": "oracle", "cpu_model": cpu_model(),
                                    "sample": f"{n} observations (every {max(cfg.num_envs // 8, 1)}th env) of this workload, all pixels, {secs:.1f} s"}
         print(json.dumps(out))
     batch.destroy()
