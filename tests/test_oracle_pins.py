@@ -315,3 +315,35 @@ def test_subpixel_offset_path_agrees_with_float_path(oracle):
     for q, (px, py) in enumerate(pxy):
         assert (sub[0][q] == full[0][py, px]).all()
         assert abs(sub[1][q] - full[1][py, px]) <= 1e-5 * max(full[1][py, px], 1e-3)
+
+
+def test_vertical_field_of_view_and_square_pixels(oracle):
+    """Square pixels: tan of the vertical half-angle is tan(hfov/2)*H/W, so on a wall at distance D the
+    pixel row py meets height cy + D*(H-1-2py)/H * (H/W) = cy + D*(H-1-2py)/W."""
+    gx, gy, gz, W, H = 8, 64, 16, 16, 8
+    grid = np.zeros((gy, gz, gx), np.uint8); grid[:, 12, :] = 1
+    cx, cy, cz = 4.5, 32.5, 2.0
+    d = _desc(oracle, grid, W, H)
+    _, depth, ids = oracle.render_obs(d, grid, None, 0, PALETTE_1, cam_row(cx, cy, cz, 0.0, 0.0))
+    for py in range(H):
+        y = cy + (12 - cz) * (H - 1 - 2 * py) / W
+        j = ids[py, W // 2, 1] // (gx * gz)
+        assert j == math.floor(y), (py, j, y)
+    assert np.allclose(depth[:, W // 2], 10.0, atol=1e-6)
+
+
+def test_tie_breaks_voxel_before_box_and_lower_box_first(oracle):
+    gx = gy = gz = 8
+    W, H = 16, 8
+    pal = np.array([[0, 0, 0], [200, 0, 0], [0, 200, 0], [0, 0, 200]], np.uint8)
+    grid = np.zeros((gy, gz, gx), np.uint8); grid[:, 6, :] = 1                      # wall face at z = 6
+    # box 0 and box 1 identical, their front face coplanar with the wall face
+    boxes = box_rows([((0, 0, 6), (8, 8, 7), 2), ((0, 0, 6), (8, 8, 7), 3)])
+    d = _desc(oracle, grid, W, H, P=4, max_boxes=2)
+    cam = cam_row(4.3, 4.2, 1.0, 0.0, 0.0)
+    rgb, depth, ids = oracle.render_obs(d, grid, boxes, 2, pal, cam)
+    c = slice(4, 12)                                                               # columns that see the wall
+    assert (ids[:, c, 0] == 0).all() and np.allclose(depth[:, c], 5.0, atol=1e-6)   # voxel wins the tie
+    rgb, depth, ids = oracle.render_obs(d, np.zeros_like(grid), boxes, 2, pal, cam)
+    assert (ids[:, c, 0] == 1).all() and (ids[:, c, 1] == 0).all()                 # lower box index wins
+    assert (rgb[:, c, 1] > 0).all() and (rgb[:, c, 2] == 0).all()                  # box 0's colour (green)
