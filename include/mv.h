@@ -108,9 +108,11 @@ typedef struct mv_body_shape {
 typedef struct mv_batch_desc {
     int32_t num_envs;                   /* N >= 1 */
     int32_t agents_per_env;             /* M >= 1 */
-    int32_t grid_x, grid_y, grid_z;     /* voxels per axis; each a multiple of 4, 4..1024;
-                                           grid_x*grid_y*grid_z/8 bytes must fit the SM's
-                                           shared memory (about 200 KiB: 1.6 M voxels) */
+    int32_t grid_x, grid_y, grid_z;     /* voxels per axis; each a multiple of 4, 4..1024.
+                                           Up to about 1.6 M voxels per env the occupancy bits
+                                           (grid_x*grid_y*grid_z/8 bytes) are staged in shared
+                                           memory; larger grids are read from global memory
+                                           (slower per step, same results) */
     int32_t max_boxes;                  /* per env, agent bodies included; 0..256 */
     int32_t width, height;              /* pixels; width a multiple of 8, height of 4; <= 4096 */
     int32_t palette_size;               /* 1..256 entries per env */
@@ -127,8 +129,8 @@ typedef struct mv_batch_desc {
 /* Allocate the device-resident world store, camera table and status word for a batch
  * (paper Section 3.2: one instance hosts N environments with M agents each).
  * desc: HOST pointer.  out: HOST pointer receiving the handle.
- * Errors: INVALID_ARG (null, out-of-range field), UNSUPPORTED (grid too large for shared
- * memory), OUT_OF_MEMORY, CUDA. */
+ * Errors: INVALID_ARG (null, out-of-range field), UNSUPPORTED (tile masks, boxes and tables of one
+ * observation exceed shared memory, e.g. a very large image), OUT_OF_MEMORY, CUDA. */
 int mv_create_batch(const mv_batch_desc *desc, mv_batch **out);
 
 /* Upload world state for envs [env_begin, env_begin+env_count) (paper Section 3.3: geometry
@@ -248,6 +250,12 @@ int mv_query_status(mv_batch *batch, int clear, void *cuda_stream);
 
 /* Number of kernels of this library launched on behalf of `batch` so far (host counter). */
 int64_t mv_launch_count(const mv_batch *batch);
+
+/* Test and measurement hook (no counterpart in the paper): on != 0 makes the render kernel read the
+ * occupancy bits from global memory instead of staging them in shared memory, which is what happens
+ * by itself for grids too large for shared memory; on == 0 restores staging (UNSUPPORTED if the grid
+ * does not fit).  Results are identical either way.  Host-only call. */
+int mv_debug_occupancy_in_global(mv_batch *batch, int on);
 
 /* Failure-detection test hook (no counterpart in the paper).  The render kernel's only device-side
  * wait is the bounded wait for the staged env block; with skip_staging != 0 the copy is not issued,

@@ -16,7 +16,7 @@ _lib = None
 MV_OK = 0
 FLAG_MATERIAL_CLAMPED, FLAG_BOX_COUNT_CLAMPED, FLAG_BAD_CAMERA, FLAG_DEVICE_TIMEOUT = 1, 2, 4, 8
 EXPORTS = ["mv_create_batch", "mv_upload_worlds", "mv_set_cameras", "mv_render_batch", "mv_step_host",
-           "mv_step_host_static", "mv_set_overlays", "mv_move_agents", "mv_merge_voxels", "mv_debug_staging", "mv_query_status", "mv_launch_count", "mv_destroy", "mv_status_string"]
+           "mv_step_host_static", "mv_set_overlays", "mv_move_agents", "mv_merge_voxels", "mv_debug_staging", "mv_debug_occupancy_in_global", "mv_query_status", "mv_launch_count", "mv_destroy", "mv_status_string"]
 
 
 class BatchDesc(C.Structure):
@@ -53,13 +53,14 @@ def lib() -> C.CDLL:
         L.mv_move_agents.argtypes = [vp, vp, vp, vp, vp]
         L.mv_merge_voxels.argtypes = [vp, i, i, vp, vp, i, vp]
         L.mv_debug_staging.argtypes = [vp, i, i]
+        L.mv_debug_occupancy_in_global.argtypes = [vp, i]
         L.mv_query_status.argtypes = [vp, i, vp]
         L.mv_launch_count.argtypes = [vp]
         L.mv_launch_count.restype = C.c_int64
         L.mv_destroy.argtypes = [vp]
         L.mv_status_string.argtypes = [i]
         L.mv_status_string.restype = C.c_char_p
-        for n in EXPORTS[:11] + ["mv_destroy"]:
+        for n in EXPORTS[:12] + ["mv_destroy"]:
             getattr(L, n).restype = i
         _lib = L
     return _lib
@@ -183,6 +184,9 @@ class Batch:
         that may not allocate GPU memory while running.  Raises MvError(-6) if the batch is too big."""
         _check(lib().mv_step_host_static(self._h, _hptr(cams, torch.int32), _hptr(rgb, torch.uint8),
                                          _hptr(depth, torch.float32), _stream(stream)), "mv_step_host_static")
+
+    def debug_occupancy_in_global(self, on: bool):
+        _check(lib().mv_debug_occupancy_in_global(self._h, int(on)), "mv_debug_occupancy_in_global")
 
     def debug_staging(self, skip_staging: bool, wait_polls: int = 1 << 18):
         _check(lib().mv_debug_staging(self._h, int(skip_staging), int(wait_polls)), "mv_debug_staging")

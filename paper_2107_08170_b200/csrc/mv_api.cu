@@ -50,6 +50,8 @@ struct mv_batch {
     int tiles_x = 0, tiles_y = 0, mask_words = 0;
     int64_t launches = 0;
     int wait_polls = 1 << 18;
+    bool occ_shared = true;             // occupancy staged in shared memory (else read from global)
+    bool occ_fits_shared = true;
     int skip_staging = 0;
     int last_cuda_error = 0;
     // mv_step_host resources (allocated on first use)
@@ -107,14 +109,19 @@ int launch_render(mv_batch *b, uint8_t *d_rgb, float *d_depth, int obs_begin, in
     p.tiles_x = b->tiles_x; p.tiles_y = b->tiles_y; p.mask_words = b->mask_words;
     p.sky_rgbx = b->sky_rgbx;
     p.miss_depth = b->desc.miss_depth;
-    p.smem_mask_off = b->smem_mask_off; p.smem_rel_off = b->smem_rel_off; p.smem_misc_off = b->smem_misc_off;
-    p.smem_ov_off = b->smem_ov_off;
+    const uint32_t unstaged = b->occ_shared ? 0u : b->lay.occ_bytes;   // shared-memory offsets shift down by it
+    p.smem_mask_off = b->smem_mask_off - unstaged; p.smem_rel_off = b->smem_rel_off - unstaged;
+    p.smem_misc_off = b->smem_misc_off - unstaged;
+    p.smem_ov_off = b->smem_ov_off - unstaged;
     p.overlay = b->d_overlay;
     p.overlay_count = b->d_overlay_count;
     p.max_overlay = b->desc.max_overlay_rects;
     p.wait_polls = b->wait_polls;
     p.skip_staging = b->skip_staging;
-    render_kernel<kRenderThreads><<<obs_count, kRenderThreads, b->smem_bytes, s>>>(p);
+    if (b->occ_shared)
+        render_kernel<kRenderThreads, true><<<obs_count, kRenderThreads, b->smem_bytes, s>>>(p);
+    else
+        render_kernel<kRenderThreads, false><<<obs_count, kRenderThreads, b->smem_bytes - b->lay.occ_bytes, s>>>(p);
     b->launches++;
     MV_CUDA(b, cudaGetLastError());
     return MV_OK;
@@ -243,9 +250,18 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
     int smem_max = 0;
     e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, d.device);
     if (e != cudaSuccess) { delete b; return MV_ERR_CUDA; }
-    if ((int)b->smem_bytes > smem_max) { delete b; return MV_ERR_UNSUPPORTED; }
-    e = cudaFuncSetAttribute(render_kernel<kRenderThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)b->smem_bytes);
+    // the occupancy normally rides in shared memory with the rest of the env block; a grid too large
+    // for that keeps it in global memory and stages only the block's tail
+    b->occ_fits_shared = (int)b->smem_bytes <= smem_max;
+    b->occ_shared = b->occ_fits_shared;
+    if ((int)(b->smem_bytes - L.occ_bytes) > smem_max) { delete b; return MV_ERR_UNSUPPORTED; }
+    e = cudaSuccess;
+    if (b->occ_fits_shared)
+        e = cudaFuncSetAttribute(render_kernel<kRenderThreads, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)b->smem_bytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(render_kernel<kRenderThreads, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(b->smem_bytes - L.occ_bytes));
     if (e != cudaSuccess) { delete b; return MV_ERR_CUDA; }
 
     const size_t blocks_bytes = (size_t)d.num_envs * L.stride;
@@ -493,6 +509,13 @@ int mv_query_status(mv_batch *b, int clear, void *cuda_stream) {
 }
 
 int64_t mv_launch_count(const mv_batch *b) { return b ? b->launches : 0; }
+
+int mv_debug_occupancy_in_global(mv_batch *b, int on) {
+    if (!b) return MV_ERR_INVALID_ARG;
+    if (!on && !b->occ_fits_shared) return MV_ERR_UNSUPPORTED;
+    b->occ_shared = !on;
+    return MV_OK;
+}
 
 int mv_debug_staging(mv_batch *b, int skip_staging, int wait_polls) {
     if (!b || wait_polls < 1 || wait_polls > (1 << 24)) return MV_ERR_INVALID_ARG;

@@ -54,8 +54,9 @@ __device__ __forceinline__ float fast_rcp(float x) {
 }
 
 // One DDA step (see the loop in render_kernel): operands %6..%8 = dt, %9..%11 = t0, %12..%14 =
-// index strides, %15 = grid-exit time, %17 = last occupancy word, %18 = shared base address.
-#define MV_DDA_STEP                                  \
+// index strides, %15 = grid-exit time, %17 = last occupancy word, %18 = shared base address
+// (or %20 = 64-bit global base address when the occupancy does not fit shared memory).
+#define MV_DDA_MOVE                                  \
     " min.f32 t, tx, ty, tz;\n"                      \
     " setp.geu.f32 pq, t, %15;\n"                    \
     " @pq bra MV_DDA_DONE;\n"                        \
@@ -72,19 +73,56 @@ __device__ __forceinline__ float fast_rcp(float x) {
     " fma.rn.f32 ty, ky, %7, %10;\n"                 \
     " fma.rn.f32 tz, kz, %8, %11;\n"                 \
     " shr.u32 a, vi, 5;\n"                           \
-    " min.u32 a, a, %17;\n"                          \
-    " shl.b32 a, a, 2;\n"                            \
-    " add.u32 a, a, %18;\n"                          \
-    " ld.shared.u32 w, [a];\n"                       \
+    " min.u32 a, a, %17;\n"
+#define MV_DDA_TEST                                  \
     " shf.r.wrap.b32 w, w, 0, vi;\n"                 \
     " and.b32 w, w, 1;\n"                            \
     " setp.ne.u32 pq, w, 0;\n"                       \
     " @pq bra MV_DDA_HIT;\n"
+#define MV_DDA_STEP MV_DDA_MOVE " shl.b32 a, a, 2;\n add.u32 a, a, %18;\n ld.shared.u32 w, [a];\n" MV_DDA_TEST
+#define MV_DDA_STEP_GLOBAL MV_DDA_MOVE " mad.wide.u32 ag, a, 4, %20;\n ld.global.nc.u32 w, [ag];\n" MV_DDA_TEST
+#define MV_DDA_PROLOGUE                              \
+    "{\n"                                            \
+    " .reg .pred px, py, pxy, pq;\n"                 \
+    " .reg .f32 t, tx, ty, tz, kx, ky, kz, th;\n"    \
+    " .reg .u32 w, a, hit;\n"                        \
+    " .reg .u64 ag;\n"                               \
+    " .reg .s32 vi, it;\n"                           \
+    " mov.f32 tx, %9;\n"                             \
+    " mov.f32 ty, %10;\n"                            \
+    " mov.f32 tz, %11;\n"                            \
+    " mov.f32 kx, 0f00000000;\n"                     \
+    " mov.f32 ky, 0f00000000;\n"                     \
+    " mov.f32 kz, 0f00000000;\n"                     \
+    " mov.f32 th, 0f00000000;\n"                     \
+    " mov.u32 hit, 0;\n"                             \
+    " mov.s32 vi, %19;\n"                            \
+    " mov.s32 it, %16;\n"                            \
+    "MV_DDA_LOOP:\n"
+#define MV_DDA_EPILOGUE                              \
+    " sub.u32 it, it, 2;\n"                          \
+    " setp.gt.s32 pq, it, 0;\n"                      \
+    " @pq bra MV_DDA_LOOP;\n"                        \
+    " bra MV_DDA_DONE;\n"                            \
+    "MV_DDA_HIT:\n"                                  \
+    " mov.f32 th, t;\n"                              \
+    " mov.u32 hit, 1;\n"                             \
+    "MV_DDA_DONE:\n"                                 \
+    " mov.f32 %0, kx;\n"                             \
+    " mov.f32 %1, ky;\n"                             \
+    " mov.f32 %2, kz;\n"                             \
+    " mov.s32 %3, vi;\n"                             \
+    " mov.f32 %4, th;\n"                             \
+    " mov.u32 %5, hit;\n"                            \
+    "}\n"
 
 #ifndef MV_MINB
 #define MV_MINB 3
 #endif
-template <int NT>
+// OCC_SHARED: the occupancy bits are staged in shared memory with the rest of the env block (the
+// normal case); otherwise only the block's tail (colour table, boxes, bounds) is staged and the
+// occupancy is read from global memory through the read-only path.
+template <int NT, bool OCC_SHARED>
 __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -93,10 +131,14 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     const int env = obs / p.agents;
     const int W = p.W, H = p.H;
 
-    const uint32_t *s_occ = reinterpret_cast<const uint32_t *>(smem);
-    const uint32_t *s_lut = reinterpret_cast<const uint32_t *>(smem + p.lay.lut_off);
-    const float4 *s_box = reinterpret_cast<const float4 *>(smem + p.lay.box_off);
-    const int *s_count = reinterpret_cast<const int *>(smem + p.lay.count_off);
+    // bytes of the env block that are NOT staged (the occupancy, when it stays in global memory)
+    const uint32_t unstaged = OCC_SHARED ? 0u : p.lay.occ_bytes;
+    const unsigned char *env_block = p.env_blocks + (size_t)env * p.lay.stride;
+    const uint32_t *s_occ = OCC_SHARED ? reinterpret_cast<const uint32_t *>(smem)
+                                       : reinterpret_cast<const uint32_t *>(env_block);
+    const uint32_t *s_lut = reinterpret_cast<const uint32_t *>(smem + (p.lay.lut_off - unstaged));
+    const float4 *s_box = reinterpret_cast<const float4 *>(smem + (p.lay.box_off - unstaged));
+    const int *s_count = reinterpret_cast<const int *>(smem + (p.lay.count_off - unstaged));
     uint32_t *s_mask = reinterpret_cast<uint32_t *>(smem + p.smem_mask_off);
     float4 *s_rel = reinterpret_cast<float4 *>(smem + p.smem_rel_off);
     uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + p.smem_misc_off);
@@ -126,8 +168,8 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     if (tid == 0) mbar_init(s_bar, 1);
     __syncthreads();
     if (tid == 0 && !p.skip_staging) {
-        mbar_expect_tx(s_bar, p.lay.block_bytes);
-        bulk_load(smem, p.env_blocks + (size_t)env * p.lay.stride, p.lay.block_bytes, s_bar);
+        mbar_expect_tx(s_bar, p.lay.block_bytes - unstaged);
+        bulk_load(smem, env_block + unstaged, p.lay.block_bytes - unstaged, s_bar);
     }
     const int ntiles = p.tiles_x * p.tiles_y;
     const int mw = p.mask_words;
@@ -327,44 +369,19 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             uint32_t hit;
             int vout;
             float th;
-            asm volatile(
-                "{\n"
-                " .reg .pred px, py, pxy, pq;\n"
-                " .reg .f32 t, tx, ty, tz, kx, ky, kz, th;\n"
-                " .reg .u32 w, a, hit;\n"
-                " .reg .s32 vi, it;\n"
-                " mov.f32 tx, %9;\n"
-                " mov.f32 ty, %10;\n"
-                " mov.f32 tz, %11;\n"
-                " mov.f32 kx, 0f00000000;\n"
-                " mov.f32 ky, 0f00000000;\n"
-                " mov.f32 kz, 0f00000000;\n"
-                " mov.f32 th, 0f00000000;\n"
-                " mov.u32 hit, 0;\n"
-                " mov.s32 vi, %19;\n"
-                " mov.s32 it, %16;\n"
-                "MV_DDA_LOOP:\n"
-                MV_DDA_STEP
-                MV_DDA_STEP
-                " sub.u32 it, it, 2;\n"
-                " setp.gt.s32 pq, it, 0;\n"
-                " @pq bra MV_DDA_LOOP;\n"
-                " bra MV_DDA_DONE;\n"
-                "MV_DDA_HIT:\n"
-                " mov.f32 th, t;\n"
-                " mov.u32 hit, 1;\n"
-                "MV_DDA_DONE:\n"
-                " mov.f32 %0, kx;\n"
-                " mov.f32 %1, ky;\n"
-                " mov.f32 %2, kz;\n"
-                " mov.s32 %3, vi;\n"
-                " mov.f32 %4, th;\n"
-                " mov.u32 %5, hit;\n"
-                "}\n"
-                : "=f"(kx), "=f"(ky), "=f"(kz), "=r"(vout), "=f"(th), "=r"(hit)
-                : "f"(dtx), "f"(dty), "f"(dtz), "f"(t0x), "f"(t0y), "f"(t0z), "r"(sx), "r"(sy), "r"(sz),
-                  "f"(t_exit), "r"((uint32_t)max_steps), "r"(last_word), "r"(smem_addr(smem)), "r"(vi)
-                : "memory");
+            if constexpr (OCC_SHARED) {
+                asm volatile(MV_DDA_PROLOGUE MV_DDA_STEP MV_DDA_STEP MV_DDA_EPILOGUE
+                             : "=f"(kx), "=f"(ky), "=f"(kz), "=r"(vout), "=f"(th), "=r"(hit)
+                             : "f"(dtx), "f"(dty), "f"(dtz), "f"(t0x), "f"(t0y), "f"(t0z), "r"(sx), "r"(sy), "r"(sz),
+                               "f"(t_exit), "r"((uint32_t)max_steps), "r"(last_word), "r"(smem_addr(smem)), "r"(vi)
+                             : "memory");
+            } else {
+                asm volatile(MV_DDA_PROLOGUE MV_DDA_STEP_GLOBAL MV_DDA_STEP_GLOBAL MV_DDA_EPILOGUE
+                             : "=f"(kx), "=f"(ky), "=f"(kz), "=r"(vout), "=f"(th), "=r"(hit)
+                             : "f"(dtx), "f"(dty), "f"(dtz), "f"(t0x), "f"(t0y), "f"(t0z), "r"(sx), "r"(sy), "r"(sz),
+                               "f"(t_exit), "r"((uint32_t)max_steps), "r"(last_word), "r"(0u), "r"(vi), "l"(s_occ)
+                             : "memory");
+            }
             vi = vout;
             if (hit) t_hit = th;
             vhit = loop_hit = hit != 0;

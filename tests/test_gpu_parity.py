@@ -309,10 +309,44 @@ def test_not_ready_and_argument_errors():
 def test_limits_are_reported_not_faulted():
     B = _binding()
     import ctypes as C
-    # occupancy of 1024 x 64 x 1024 voxels is 8 MiB: far beyond shared memory -> UNSUPPORTED, no launch
-    d = B.make_desc(1, 1, (1024, 64, 1024), 0, 64, 36, 16)
+    # per-observation tables (tile masks of a 4096 x 4096 image) beyond shared memory -> UNSUPPORTED, no launch
+    d = B.make_desc(1, 1, (16, 8, 16), 32, 4096, 4096, 16)
     h = C.c_void_p()
     assert B.lib().mv_create_batch(C.byref(d), C.byref(h)) == -6 and not h.value
+
+
+def test_occupancy_in_global_memory_matches_shared(oracle):
+    """Grids too large for shared memory are walked in global memory; forcing that path on an
+    ordinary workload gives the same bytes, and a grid that really is too large matches the oracle."""
+    from gpu_util import upload_scene, scene_to_numpy
+    B = _binding()
+    cfg = scenes.config("rooms_boxes", num_envs=4)
+    sc = scenes.make_scene(cfg)
+    batch = B.Batch(B.desc_from_config(cfg))
+    upload_scene(batch, sc)
+    batch.set_cameras(sc["cams"].cuda())
+    rgb, depth = batch.alloc_outputs()
+    batch.render_batch(rgb, depth)
+    rgb2, depth2 = batch.alloc_outputs()
+    batch.debug_occupancy_in_global(True)
+    batch.render_batch(rgb2, depth2)
+    assert torch.equal(rgb, rgb2) and torch.equal(depth, depth2) and batch.query_status() == 0
+    batch.debug_occupancy_in_global(False)
+    batch.destroy()
+    # 256 x 32 x 256 voxels: 256 KiB of occupancy bits per env, more than an SM's shared memory
+    big = scenes.config("headline", num_envs=2, grid=(256, 32, 256), width=64, height=36, extra={"n_rects": 4200})
+    sb = scenes.make_scene(big)
+    bb = B.Batch(B.desc_from_config(big))
+    with pytest.raises(B.MvError):
+        bb.debug_occupancy_in_global(False)              # cannot be staged
+    upload_scene(bb, sb)
+    bb.set_cameras(sb["cams"].cuda())
+    r, d = bb.alloc_outputs()
+    bb.render_batch(r, d)
+    assert bb.query_status() == 0
+    st = parity.compare_scene(oracle, big, scene_to_numpy(sb), range(big.num_obs), r.cpu().numpy(), d.cpu().numpy())
+    parity.assert_parity(st, "large grid")
+    bb.destroy()
 
 
 def test_odd_grid_sizes_and_occupied_bounds(oracle):
