@@ -207,7 +207,10 @@ def main():
     assert torch.cuda.is_available(), "bench.py needs a CUDA device"
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
+    # under torchrun (RANK set) the process group is used even for one rank, so the single-GPU launch
+    # exercises the same barrier and max-over-ranks code as the multi-GPU one
+    use_dist = world > 1 or ("RANK" in os.environ and "MASTER_ADDR" in os.environ)
+    if use_dist:
         dist.init_process_group("nccl", device_id=dev)
 
     cfg = scenes.config(WORKLOAD) if args.envs is None else scenes.config(WORKLOAD, num_envs=args.envs)
@@ -217,7 +220,7 @@ def main():
     stream = torch.cuda.current_stream()
 
     def barrier():
-        if world > 1:
+        if use_dist:
             dist.barrier()
         torch.cuda.synchronize(dev)
 
@@ -327,7 +330,7 @@ def main():
                                    "sample": f"{n} observations (every {max(cfg.num_envs // 8, 1)}th env) of this workload, all pixels, {secs:.1f} s"}
         print(json.dumps(out))
     batch.destroy()
-    if world > 1:
+    if use_dist:
         dist.destroy_process_group()
 
 

@@ -22,6 +22,6 @@ def split_envs(total_envs: int, rank: int, world: int):
 def max_over_ranks(values, device):
     """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
     t = torch.tensor(list(values), dtype=torch.float64, device=device)
-    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+    if dist.is_available() and dist.is_initialized():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return [float(x) for x in t]
