@@ -131,6 +131,44 @@ def cpu_oracle_rate(cfg, kept, max_seconds=25.0, max_obs=8):
     return done / dt, done, dt, mv_oracle.threads_used()
 
 
+def time_extras(batch, cfg, cams, rgb, depth, dev):
+    """CUDA-event medians (ms) of the entry points beside the render step, on the benchmark's batch."""
+    import torch
+    from paper_2107_08170_b200 import vecenv
+
+    def med(fn, n=15):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize(dev)
+        ts = []
+        for _ in range(n):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record(); torch.cuda.synchronize(dev)
+            ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts)
+
+    out = {"render_ms": med(lambda: batch.render_batch(rgb, depth))}
+    E = cfg.num_envs
+    rects = vecenv.time_bar_rects(torch.full((E,), 60), torch.full((E,), 100), cfg.width, cfg.agents).to(dev)
+    count = torch.ones(cfg.num_obs, dtype=torch.int32, device=dev)
+    out["set_overlays_ms"] = med(lambda: batch.set_overlays(rects, count))
+    out["render_with_time_bar_ms"] = med(lambda: batch.render_batch(rgb, depth))
+    batch.set_overlays(None, None)
+    moved = cams.clone()
+    yf = moved[:, 1].contiguous().view(torch.float32)
+    moved[:, 1] = (yf.floor() + 0.75).view(torch.int32)             # feet on the surface
+    moves = ((torch.rand(cfg.num_obs, 4, device=dev) - 0.5) * torch.tensor([0.4, 0.2, 0.3, 0.1], device=dev)).contiguous()
+    out["move_agents_ms"] = med(lambda: batch.move_agents(moved, moves))
+    out["set_cameras_ms"] = med(lambda: batch.set_cameras(cams))
+    n = min(E, 2048)
+    out["merge_voxels_ms_per_env"] = med(lambda: batch.merge_voxels(0, n, 2048), 3) / n
+    out["merged_boxes_per_env"] = float(batch.merge_voxels(0, n, 2048)[1].float().mean())
+    batch.debug_occupancy_in_global(True)
+    out["render_occupancy_in_global_ms"] = med(lambda: batch.render_batch(rgb, depth))
+    batch.debug_occupancy_in_global(False)
+    return out
+
+
 def run_reference(args, rank):
     """The oracle timed on a bounded sample: each step renders `sample` observations."""
     if rank != 0:
@@ -189,6 +227,8 @@ def main():
     ap.add_argument("--envs", type=int, default=None, help="override envs per GPU (profiling small cases)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--extras", action="store_true",
+                    help="also time the overlay, agent-motion and voxel-merge entry points (adds an \"extras\" object)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" and args.envs is None else args.warmup
 
@@ -215,7 +255,8 @@ def main():
 
     cfg = scenes.config(WORKLOAD) if args.envs is None else scenes.config(WORKLOAD, num_envs=args.envs)
     keep = list(range(0, cfg.num_envs, max(cfg.num_envs // 8, 1)))[:8] if rank == 0 and not args.no_cpu else []
-    batch, cams, kept = workload.build_batch(cfg, local, env_offset=shard.env_offset(rank, cfg.num_envs), keep_envs=keep)
+    batch, cams, kept = workload.build_batch(cfg, local, env_offset=shard.env_offset(rank, cfg.num_envs), keep_envs=keep,
+                                             max_overlay_rects=1 if args.extras else 0)
     rgb, depth = batch.alloc_outputs()
     stream = torch.cuda.current_stream()
 
@@ -329,6 +370,8 @@ def main():
             out["cpu_baseline"] = {"value": rate, "unit": "obs/s", "cores": cores, "kind": "oracle", "cpu_model": cpu_model(),
                                    "sample": f"{n} observations (every {max(cfg.num_envs // 8, 1)}th env) of this workload, all pixels, {secs:.1f} s"}
         print(json.dumps(out))
+    if args.extras and rank == 0:
+        print(json.dumps({"extras": time_extras(batch, cfg, cams, rgb, depth, dev)}), file=sys.stderr)
     batch.destroy()
     if use_dist:
         dist.destroy_process_group()

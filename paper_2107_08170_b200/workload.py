@@ -17,11 +17,12 @@ def algorithmic_bytes(cfg) -> int:
     return cfg.num_obs * (7 * px + 64 + px) + cfg.num_envs * (gx * gy * gz // 8 + 32 * cfg.max_boxes)
 
 
-def build_batch(cfg, device: int = 0, env_offset: int = 0, keep_envs=(), chunk_envs: int = 512):
+def build_batch(cfg, device: int = 0, env_offset: int = 0, keep_envs=(), chunk_envs: int = 512,
+                max_overlay_rects: int = 0):
     """Returns (batch, cams_dev, kept) where kept[e] holds CPU arrays of env e (local index)
     for every e in keep_envs.  env_offset shifts the seeded env ids (one range per rank)."""
     dev = torch.device("cuda", device)
-    batch = binding.Batch(binding.desc_from_config(cfg, device))
+    batch = binding.Batch(binding.desc_from_config(cfg, device, max_overlay_rects))
     cams = torch.empty(cfg.num_obs, 6, dtype=torch.int32, device=dev)
     kept = {}
     keep = set(int(e) for e in keep_envs)
