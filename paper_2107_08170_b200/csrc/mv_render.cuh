@@ -10,6 +10,9 @@
 // in shared memory, tests the tile's candidate boxes with slab tests, looks the colour up in
 // the shaded table and the warp writes 24-byte RGB row segments as packed 32-bit words and
 // 32-byte depth row segments.
+// The walk is confined to the cell box that holds every filled voxel of the environment (built at
+// upload), so rays that leave it stop at once; GUI rectangles, if any, are painted over the colour
+// just before the store.
 #pragma once
 #include "mv_device.cuh"
 
