@@ -413,3 +413,36 @@ def test_translation_and_occlusion_invariants_on_gpu(oracle):
     r0 = _render_custom(oracle, g, pal3, cam, W, H, boxes=hidden, box_count=np.array([0]), max_boxes=1, check=False)
     r1 = _render_custom(oracle, g2, pal3, cam, W, H, boxes=hidden, box_count=np.array([1]), max_boxes=1, check=False)
     assert (r0[0] == r1[0]).all() and (r0[1] == r1[1]).all()
+
+
+def test_fuzz_cameras_anywhere_with_boxes(oracle):
+    """Random small worlds, cameras inside, outside, high above and inside solids, random boxes."""
+    rng = np.random.default_rng(99)
+    E, A, gx, gy, gz, W, H, nb = 24, 2, 16, 8, 12, 64, 36, 6
+    grid = ((rng.random((E, gy, gz, gx)) < rng.uniform(0.02, 0.35, size=(E, 1, 1, 1))) *
+            rng.integers(1, 8, size=(E, gy, gz, gx))).astype(np.uint8)
+    grid[::3, 0] = 1
+    grid[5] = 0                                                  # an empty world
+    pal = _pal(E, 8, seed=4)
+    boxes = np.zeros((E, nb, 8), np.int32)
+    for e in range(E):
+        rows = []
+        for b in range(nb):
+            c = rng.uniform([-3, -2, -3], [gx + 3, gy + 2, gz + 3]); s = rng.uniform(0.2, 3.0, 3)
+            rows.append((c - s / 2, c + s / 2, int(rng.integers(0, 8))))
+        boxes[e] = box_rows(rows)
+    count = rng.integers(0, nb + 1, size=E)
+    cams = []
+    for o in range(E * A):
+        pos = rng.uniform([-6, -4, -6], [gx + 6, gy + 6, gz + 6])
+        if o % 4 == 0:
+            pos = rng.uniform([0.5, 0.5, 0.5], [gx - 0.5, gy - 0.5, gz - 0.5])
+        tgt = np.array([gx / 2, gy / 2, gz / 2]) + rng.normal(0, 3, 3)
+        v = tgt - pos
+        yaw = math.atan2(v[0], v[2]); pitch = math.atan2(v[1], math.hypot(v[0], v[2]))
+        cams.append(cam_row(*pos, yaw, float(np.clip(pitch, -1.4, 1.4)), self_box=int(rng.integers(-1, nb))))
+    g_rgb, g_depth, status, st = _render_custom(oracle, grid, pal, np.stack(cams), W, H, boxes=boxes,
+                                                box_count=count, agents=A, max_boxes=nb)
+    assert status == 0
+    parity.assert_parity(st, "fuzz")
+    assert st["pixels"] == E * A * W * H and (g_depth > 0).mean() > 0.2
