@@ -314,9 +314,11 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         const float ix = fast_rcp(dx), iy = fast_rcp(dy), iz = fast_rcp(dz);
         const bool ngx = dx < 0.0f, ngy = dy < 0.0f, ngz = dz < 0.0f;
         const float dtx = fabsf(ix), dty = fabsf(iy), dtz = fabsf(iz);
-        const float4 qx = s_dda[0 + (__float_as_uint(dx) >> 31)];
-        const float4 qy = s_dda[2 + (__float_as_uint(dy) >> 31)];
-        const float4 qz = s_dda[4 + (__float_as_uint(dz) >> 31)];
+        const uint32_t bx_ = __float_as_uint(dx) >> 31, by_ = __float_as_uint(dy) >> 31, bz_ = __float_as_uint(dz) >> 31;
+        const uint32_t sgn3 = bx_ | (by_ << 1) | (bz_ << 2);        // bit c set: component c negative
+        const float4 qx = s_dda[0 + bx_];
+        const float4 qy = s_dda[2 + by_];
+        const float4 qz = s_dda[4 + bz_];
         const int sx = __float_as_int(qx.z), sy = __float_as_int(qy.z), sz = __float_as_int(qz.z);
 
         // ---- grid traversal: crossing times are t0 + k*dt with integer-valued k, so the exit
@@ -419,8 +421,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                         tb = t;
                         bmat = __float_as_uint(hi.w);
                         const int ax = (nx == tn) ? 0 : ((ny == tn) ? 1 : 2);
-                        const float ds = ax == 0 ? dx : (ax == 1 ? dy : dz);
-                        bface = (tn < 0.0f) ? kFaceInside : 2 * ax + (ds > 0.0f ? 0 : 1);
+                        bface = (tn < 0.0f) ? kFaceInside : 2 * ax + (int)((sgn3 >> ax) & 1u);
                     }
                 }
             }
@@ -434,8 +435,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             depth = tb + 0.0f;
         } else if (vhit) {
             const int m = __ldg(mat_env + vi);
-            const float ds = axis == 0 ? dx : (axis == 1 ? dy : dz);
-            const int face = axis < 0 ? kFaceInside : 2 * axis + (ds > 0.0f ? 0 : 1);
+            const int face = axis < 0 ? kFaceInside : 2 * axis + (int)((sgn3 >> axis) & 1u);
             rgbx = s_lut[face * P_ + m];
             depth = t_hit + 0.0f;
         }
