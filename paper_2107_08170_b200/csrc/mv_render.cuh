@@ -56,34 +56,34 @@ __device__ __forceinline__ float fast_rcp(float x) {
     return r;
 }
 
-// One DDA step (see the loop in render_kernel): operands %6..%8 = dt, %9..%11 = t0, %12..%14 =
-// index strides, %15 = grid-exit time, %17 = last occupancy word, %18 = shared base address
-// (or %20 = 64-bit global base address when the occupancy does not fit shared memory).
+// One DDA step (see the loop in render_kernel): operands %3..%5 = dt, %6..%8 = t0, %9..%11 =
+// index strides, %12 = grid-exit time, %14 = last occupancy word, %15 = shared base address
+// (or %17 = 64-bit global base address when the occupancy does not fit shared memory).
 #define MV_DDA_MOVE                                  \
     " min.f32 t, tx, ty, tz;\n"                      \
-    " setp.geu.f32 pq, t, %15;\n"                    \
+    " setp.geu.f32 pq, t, %12;\n"                    \
     " @pq bra MV_DDA_DONE;\n"                        \
     " setp.eq.f32 px, tx, t;\n"                      \
     " setp.eq.and.f32 py, ty, t, !px;\n"             \
     " or.pred pxy, px, py;\n"                        \
     " @px add.f32 kx, kx, 0f3F800000;\n"             \
-    " @px add.s32 vi, vi, %12;\n"                    \
+    " @px add.s32 vi, vi, %9;\n"                    \
     " @py add.f32 ky, ky, 0f3F800000;\n"             \
-    " @py add.s32 vi, vi, %13;\n"                    \
+    " @py add.s32 vi, vi, %10;\n"                    \
     " @!pxy add.f32 kz, kz, 0f3F800000;\n"           \
-    " @!pxy add.s32 vi, vi, %14;\n"                  \
-    " fma.rn.f32 tx, kx, %6, %9;\n"                  \
-    " fma.rn.f32 ty, ky, %7, %10;\n"                 \
-    " fma.rn.f32 tz, kz, %8, %11;\n"                 \
+    " @!pxy add.s32 vi, vi, %11;\n"                  \
+    " fma.rn.f32 tx, kx, %3, %6;\n"                  \
+    " fma.rn.f32 ty, ky, %4, %7;\n"                 \
+    " fma.rn.f32 tz, kz, %5, %8;\n"                 \
     " shr.u32 a, vi, 5;\n"                           \
-    " min.u32 a, a, %17;\n"
+    " min.u32 a, a, %14;\n"
 #define MV_DDA_TEST                                  \
     " shf.r.wrap.b32 w, w, 0, vi;\n"                 \
     " and.b32 w, w, 1;\n"                            \
     " setp.ne.u32 pq, w, 0;\n"                       \
     " @pq bra MV_DDA_HIT;\n"
-#define MV_DDA_STEP MV_DDA_MOVE " shl.b32 a, a, 2;\n add.u32 a, a, %18;\n ld.shared.u32 w, [a];\n" MV_DDA_TEST
-#define MV_DDA_STEP_GLOBAL MV_DDA_MOVE " mad.wide.u32 ag, a, 4, %20;\n ld.global.nc.u32 w, [ag];\n" MV_DDA_TEST
+#define MV_DDA_STEP MV_DDA_MOVE " shl.b32 a, a, 2;\n add.u32 a, a, %15;\n ld.shared.u32 w, [a];\n" MV_DDA_TEST
+#define MV_DDA_STEP_GLOBAL MV_DDA_MOVE " mad.wide.u32 ag, a, 4, %17;\n ld.global.nc.u32 w, [ag];\n" MV_DDA_TEST
 #define MV_DDA_PROLOGUE                              \
     "{\n"                                            \
     " .reg .pred px, py, pxy, pq;\n"                 \
@@ -91,16 +91,16 @@ __device__ __forceinline__ float fast_rcp(float x) {
     " .reg .u32 w, a, hit;\n"                        \
     " .reg .u64 ag;\n"                               \
     " .reg .s32 vi, it;\n"                           \
-    " mov.f32 tx, %9;\n"                             \
-    " mov.f32 ty, %10;\n"                            \
-    " mov.f32 tz, %11;\n"                            \
+    " mov.f32 tx, %6;\n"                             \
+    " mov.f32 ty, %7;\n"                            \
+    " mov.f32 tz, %8;\n"                            \
     " mov.f32 kx, 0f00000000;\n"                     \
     " mov.f32 ky, 0f00000000;\n"                     \
     " mov.f32 kz, 0f00000000;\n"                     \
     " mov.f32 th, 0f00000000;\n"                     \
     " mov.u32 hit, 0;\n"                             \
-    " mov.s32 vi, %19;\n"                            \
-    " mov.s32 it, %16;\n"                            \
+    " mov.s32 vi, %16;\n"                            \
+    " mov.s32 it, %13;\n"                            \
     "MV_DDA_LOOP:\n"
 #define MV_DDA_EPILOGUE                              \
     " sub.u32 it, it, 2;\n"                          \
@@ -109,14 +109,12 @@ __device__ __forceinline__ float fast_rcp(float x) {
     " bra MV_DDA_DONE;\n"                            \
     "MV_DDA_HIT:\n"                                  \
     " mov.f32 th, t;\n"                              \
-    " mov.u32 hit, 1;\n"                             \
+    " selp.u32 hit, 2, 3, py;\n"                     \
+    " selp.u32 hit, 1, hit, px;\n"                   \
     "MV_DDA_DONE:\n"                                 \
-    " mov.f32 %0, kx;\n"                             \
-    " mov.f32 %1, ky;\n"                             \
-    " mov.f32 %2, kz;\n"                             \
-    " mov.s32 %3, vi;\n"                             \
-    " mov.f32 %4, th;\n"                             \
-    " mov.u32 %5, hit;\n"                            \
+    " mov.s32 %0, vi;\n"                             \
+    " mov.f32 %1, th;\n"                             \
+    " mov.u32 %2, hit;\n"                            \
     "}\n"
 
 #ifndef MV_MINB
@@ -360,8 +358,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             vhit = alive && ((s_occ[vi >> 5] >> (vi & 31)) & 1u);
             if (!alive) t_exit = -kInf;
         }
-        float kx = 0.0f, ky = 0.0f, kz = 0.0f;
-        bool loop_hit = false;
+        int loop_axis = 0;
         if (!vhit) {
             // 3D-DDA written in PTX so that each step is a fixed short sequence of predicated
             // instructions: t = min(tx,ty,tz); stop when t >= t_exit; step the axis whose crossing
@@ -376,27 +373,26 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             float th;
             if constexpr (OCC_SHARED) {
                 asm volatile(MV_DDA_PROLOGUE MV_DDA_STEP MV_DDA_STEP MV_DDA_EPILOGUE
-                             : "=f"(kx), "=f"(ky), "=f"(kz), "=r"(vout), "=f"(th), "=r"(hit)
+                             : "=r"(vout), "=f"(th), "=r"(hit)
                              : "f"(dtx), "f"(dty), "f"(dtz), "f"(t0x), "f"(t0y), "f"(t0z), "r"(sx), "r"(sy), "r"(sz),
                                "f"(t_exit), "r"((uint32_t)max_steps), "r"(last_word), "r"(smem_addr(smem)), "r"(vi)
                              : "memory");
             } else {
                 asm volatile(MV_DDA_PROLOGUE MV_DDA_STEP_GLOBAL MV_DDA_STEP_GLOBAL MV_DDA_EPILOGUE
-                             : "=f"(kx), "=f"(ky), "=f"(kz), "=r"(vout), "=f"(th), "=r"(hit)
+                             : "=r"(vout), "=f"(th), "=r"(hit)
                              : "f"(dtx), "f"(dty), "f"(dtz), "f"(t0x), "f"(t0y), "f"(t0z), "r"(sx), "r"(sy), "r"(sz),
                                "f"(t_exit), "r"((uint32_t)max_steps), "r"(last_word), "r"(0u), "r"(vi), "l"(s_occ)
                              : "memory");
             }
             vi = vout;
             if (hit) t_hit = th;
-            vhit = loop_hit = hit != 0;
+            vhit = hit != 0;
+            loop_axis = (int)hit;
         }
         __syncwarp();
-        // entered face: the axis whose crossing time equals the hit time (z, y, x order undoes the
-        // tie order of the steps); no step taken = the grid-entry axis, or none = eye inside a solid
-        int axis = axis0;
-        if (loop_hit)
-            axis = fmaf(kz - 1.0f, dtz, t0z) == t_hit ? 2 : (fmaf(ky - 1.0f, dty, t0y) == t_hit ? 1 : 0);
+        // entered face: the axis of the last step (the loop reports 1 + axis at a hit), else the
+        // box-entry axis, else none = eye inside a solid
+        const int axis = loop_axis > 0 ? loop_axis - 1 : axis0;
 
         // ---- boxes of this tile (skip those wholly behind every lane's voxel hit)
         float tb = kInf;
