@@ -251,19 +251,32 @@ int mv_query_status(mv_batch *batch, int clear, void *cuda_stream);
 /* Number of kernels of this library launched on behalf of `batch` so far (host counter). */
 int64_t mv_launch_count(const mv_batch *batch);
 
-/* Test and measurement hook (no counterpart in the paper): on != 0 makes the render kernel read the
- * occupancy bits from global memory instead of staging them in shared memory, which is what happens
- * by itself for grids too large for shared memory; on == 0 restores staging (UNSUPPORTED if the grid
- * does not fit).  Results are identical either way.  Host-only call. */
+/* ---- Test and measurement hooks (no counterpart in the paper).  They are exported by the library but
+ * declared only for translation units that define MV_ENABLE_TEST_HOOKS before including this header;
+ * they change how the render kernel runs, never what it computes.  Host-only calls. */
+#ifdef MV_ENABLE_TEST_HOOKS
+
+/* on != 0 makes the render kernel read the occupancy bits from global memory instead of staging them
+ * in shared memory, which is what happens by itself for grids too large for shared memory; on == 0
+ * restores staging (UNSUPPORTED if the grid does not fit).  Results are identical either way. */
 int mv_debug_occupancy_in_global(mv_batch *batch, int on);
 
-/* Failure-detection test hook (no counterpart in the paper).  The render kernel's only device-side
- * wait is the bounded wait for the staged env block; with skip_staging != 0 the copy is not issued,
- * so every CTA's wait runs out after wait_polls polls, the kernel returns without touching the
- * outputs and MV_FLAG_DEVICE_TIMEOUT is set (mv_query_status then returns MV_ERR_DEVICE_TIMEOUT).
- * Nothing faults or hangs and the context stays usable.  Defaults: skip_staging 0, wait_polls
- * 2^18; wait_polls must be in 1..2^24.  Host-only call.  Errors: INVALID_ARG. */
+/* Failure-detection hook.  The render kernel's only device-side wait is the bounded wait for the
+ * staged env block; with skip_staging != 0 the copy is not issued, so every CTA's wait runs out after
+ * wait_polls polls, the kernel returns without touching the outputs and MV_FLAG_DEVICE_TIMEOUT is set
+ * (mv_query_status then returns MV_ERR_DEVICE_TIMEOUT).  Nothing faults or hangs and the context stays
+ * usable.  Defaults: skip_staging 0, wait_polls 2^18; wait_polls must be in 1..2^24.
+ * Errors: INVALID_ARG. */
 int mv_debug_staging(mv_batch *batch, int skip_staging, int wait_polls);
+
+/* How many observations one CTA of the render kernel renders: 1 (a CTA per observation) or
+ * agents_per_env (a CTA per environment, its block staged once for all its agents); 0 restores the
+ * library's own choice, which depends on how many environments the batch has.  Results are identical.
+ * Errors: INVALID_ARG (any other value), UNSUPPORTED (the per-environment shape does not fit shared
+ * memory). */
+int mv_debug_agents_per_cta(mv_batch *batch, int agents_per_cta);
+
+#endif /* MV_ENABLE_TEST_HOOKS */
 
 /* Free everything mv_create_batch allocated (synchronises the device). NULL is accepted. */
 int mv_destroy(mv_batch *batch);

@@ -16,7 +16,7 @@ _lib = None
 MV_OK = 0
 FLAG_MATERIAL_CLAMPED, FLAG_BOX_COUNT_CLAMPED, FLAG_BAD_CAMERA, FLAG_DEVICE_TIMEOUT = 1, 2, 4, 8
 EXPORTS = ["mv_create_batch", "mv_upload_worlds", "mv_set_cameras", "mv_render_batch", "mv_step_host",
-           "mv_step_host_static", "mv_set_overlays", "mv_move_agents", "mv_merge_voxels", "mv_debug_staging", "mv_debug_occupancy_in_global", "mv_query_status", "mv_launch_count", "mv_destroy", "mv_status_string"]
+           "mv_step_host_static", "mv_set_overlays", "mv_move_agents", "mv_merge_voxels", "mv_debug_staging", "mv_debug_occupancy_in_global", "mv_debug_agents_per_cta", "mv_query_status", "mv_launch_count", "mv_destroy", "mv_status_string"]
 
 
 class BatchDesc(C.Structure):
@@ -54,13 +54,14 @@ def lib() -> C.CDLL:
         L.mv_merge_voxels.argtypes = [vp, i, i, vp, vp, i, vp]
         L.mv_debug_staging.argtypes = [vp, i, i]
         L.mv_debug_occupancy_in_global.argtypes = [vp, i]
+        L.mv_debug_agents_per_cta.argtypes = [vp, i]
         L.mv_query_status.argtypes = [vp, i, vp]
         L.mv_launch_count.argtypes = [vp]
         L.mv_launch_count.restype = C.c_int64
         L.mv_destroy.argtypes = [vp]
         L.mv_status_string.argtypes = [i]
         L.mv_status_string.restype = C.c_char_p
-        for n in EXPORTS[:12] + ["mv_destroy"]:
+        for n in [e for e in EXPORTS if e not in ("mv_launch_count", "mv_status_string")]:
             getattr(L, n).restype = i
         _lib = L
     return _lib
@@ -187,6 +188,10 @@ class Batch:
 
     def debug_occupancy_in_global(self, on: bool):
         _check(lib().mv_debug_occupancy_in_global(self._h, int(on)), "mv_debug_occupancy_in_global")
+
+    def debug_agents_per_cta(self, agents_per_cta: int):
+        """1 = a CTA per observation, agents_per_env = a CTA per environment, 0 = the library's choice."""
+        _check(lib().mv_debug_agents_per_cta(self._h, int(agents_per_cta)), "mv_debug_agents_per_cta")
 
     def debug_staging(self, skip_staging: bool, wait_polls: int = 1 << 18):
         _check(lib().mv_debug_staging(self._h, int(skip_staging), int(wait_polls)), "mv_debug_staging")

@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in include/mv.h: argument checks, allocation of the
 // device-resident world store, and the kernel launches.  No rendering arithmetic runs here.
+#define MV_ENABLE_TEST_HOOKS
 #include "../../include/mv.h"
 #include "mv_device.cuh"
 #include "mv_pack.cuh"
@@ -20,6 +21,7 @@ namespace {
 #endif
 constexpr int kRenderThreads = MV_NT;
 constexpr int kHostChunks = 8;
+constexpr double kCtaFixedCost = 0.15;   // staging + set-up of a CTA, in units of one observation's render time
 constexpr size_t kMergeScratchBytes = 256u << 20;   // coverage bitmap for the envs of one merge launch
 
 inline uint32_t round_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
@@ -39,19 +41,22 @@ struct mv_batch {
     int merge_chunk = 0;
     int4 *d_overlay = nullptr;          // [O][max_overlay_rects]
     int32_t *d_overlay_count = nullptr; // [O]
-    uint32_t smem_ov_off = 0;
     // host-side readiness tracking (per env)
     std::vector<uint8_t> has_grid, has_palette;
     int missing_grid = 0, missing_palette = 0;
     bool has_cams = false;
     double kr = 0, ku = 0;
     uint32_t sky_rgbx = 0;
-    uint32_t smem_mask_off = 0, smem_rel_off = 0, smem_misc_off = 0, smem_bytes = 0;
+    struct Smem { uint32_t tile_off, mask_off, rel_off, agent_off, misc_off, ov_off, bytes; };
+    Smem smem{};                        // shared-memory layout of the render kernel for agents_per_cta
+    int agents_per_cta = 1;             // observations one CTA renders: 1, or every agent of its env
     int tiles_x = 0, tiles_y = 0, mask_words = 0;
     int64_t launches = 0;
     int wait_polls = 1 << 18;
     bool occ_shared = true;             // occupancy staged in shared memory (else read from global)
     bool occ_fits_shared = true;
+    int smem_max = 0;                   // opt-in shared memory per CTA of the device
+    int auto_agents_per_cta = 1;        // the library's own choice (a test hook can override it)
     int skip_staging = 0;
     int last_cuda_error = 0;
     // mv_step_host resources (allocated on first use)
@@ -63,6 +68,7 @@ struct mv_batch {
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_chunk[kHostChunks] = {};
     cudaEvent_t ev_done = nullptr;
+    bool host_ready = false;
 };
 
 namespace {
@@ -90,6 +96,24 @@ struct DeviceGuard {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Shared-memory layout of the render kernel when one CTA renders `apc` observations of an env:
+// staged env block, tile table, then per-agent box masks, eye-relative boxes, camera records and
+// DDA start tables, the barrier and flag words, and per-agent overlay rectangles + touched-tile bits.
+mv_batch::Smem smem_layout(const mv_batch *b, int apc) {
+    const mv_batch_desc &d = b->desc;
+    const uint32_t ntiles = (uint32_t)(b->tiles_x * b->tiles_y), a = (uint32_t)apc;
+    mv_batch::Smem m{};
+    m.tile_off = round_up(b->lay.block_bytes, 16);
+    m.mask_off = m.tile_off + ntiles * 16;
+    m.rel_off = m.mask_off + round_up(a * ntiles * (uint32_t)b->mask_words * 4, 16);
+    m.agent_off = m.rel_off + a * (uint32_t)(d.max_boxes > 0 ? d.max_boxes : 1) * 32;
+    m.misc_off = m.agent_off + a * (uint32_t)(kAgentRecVecs + kDdaVecs) * 16;
+    m.ov_off = m.misc_off + 16;
+    m.bytes = m.ov_off + a * (uint32_t)(d.max_overlay_rects > 0 ? d.max_overlay_rects : 1) * 32 +
+              round_up(a * ((ntiles + 31) / 32) * 4, 16);
+    return m;
+}
+
 int launch_render(mv_batch *b, uint8_t *d_rgb, float *d_depth, int obs_begin, int obs_count, cudaStream_t s) {
     RenderParams p{};
     p.env_blocks = b->d_env_blocks;
@@ -110,18 +134,23 @@ int launch_render(mv_batch *b, uint8_t *d_rgb, float *d_depth, int obs_begin, in
     p.sky_rgbx = b->sky_rgbx;
     p.miss_depth = b->desc.miss_depth;
     const uint32_t unstaged = b->occ_shared ? 0u : b->lay.occ_bytes;   // shared-memory offsets shift down by it
-    p.smem_mask_off = b->smem_mask_off - unstaged; p.smem_rel_off = b->smem_rel_off - unstaged;
-    p.smem_misc_off = b->smem_misc_off - unstaged;
-    p.smem_ov_off = b->smem_ov_off - unstaged;
+    p.smem_tile_off = b->smem.tile_off - unstaged; p.smem_mask_off = b->smem.mask_off - unstaged;
+    p.smem_rel_off = b->smem.rel_off - unstaged; p.smem_agent_off = b->smem.agent_off - unstaged;
+    p.smem_misc_off = b->smem.misc_off - unstaged; p.smem_ov_off = b->smem.ov_off - unstaged;
+    p.agents_per_cta = b->agents_per_cta;
+    p.max_steps = b->desc.grid_x + b->desc.grid_y + b->desc.grid_z + 3;
+    // accumulated crossing times drift from the exact products by at most one rounding per step
+    p.exit_scale = 1.0f - (float)(b->desc.grid_x + b->desc.grid_y + b->desc.grid_z + 3) * 1.1920929e-7f;
     p.overlay = b->d_overlay;
     p.overlay_count = b->d_overlay_count;
     p.max_overlay = b->desc.max_overlay_rects;
     p.wait_polls = b->wait_polls;
     p.skip_staging = b->skip_staging;
+    const int ctas = obs_count / b->agents_per_cta;   // callers pass whole environments when a CTA renders one
     if (b->occ_shared)
-        render_kernel<kRenderThreads, true><<<obs_count, kRenderThreads, b->smem_bytes, s>>>(p);
+        render_kernel<kRenderThreads, true><<<ctas, kRenderThreads, b->smem.bytes, s>>>(p);
     else
-        render_kernel<kRenderThreads, false><<<obs_count, kRenderThreads, b->smem_bytes - b->lay.occ_bytes, s>>>(p);
+        render_kernel<kRenderThreads, false><<<ctas, kRenderThreads, b->smem.bytes - b->lay.occ_bytes, s>>>(p);
     b->launches++;
     MV_CUDA(b, cudaGetLastError());
     return MV_OK;
@@ -146,6 +175,50 @@ int launch_boxes(mv_batch *b, int env_begin, int env_count, const mv_box *d_boxe
     b->launches++;
     MV_CUDA(b, cudaGetLastError());
     return MV_OK;
+}
+
+// First-use resources of mv_step_host: all of them or none, so that a failed attempt can be retried.
+void free_host_step(mv_batch *b) {
+    cudaFree(b->d_rgb); cudaFree(b->d_depth); cudaFree(b->d_cam_in); cudaFree(b->d_box_in); cudaFree(b->d_count_in);
+    b->d_rgb = nullptr; b->d_depth = nullptr; b->d_cam_in = nullptr; b->d_box_in = nullptr; b->d_count_in = nullptr;
+    if (b->copy_stream) cudaStreamDestroy(b->copy_stream);
+    b->copy_stream = nullptr;
+    for (auto &ev : b->ev_chunk) { if (ev) cudaEventDestroy(ev); ev = nullptr; }
+    if (b->ev_done) cudaEventDestroy(b->ev_done);
+    b->ev_done = nullptr;
+    b->host_ready = false;
+}
+
+int alloc_host_step(mv_batch *b) {
+    const size_t px = (size_t)b->desc.width * b->desc.height;
+    const size_t O = (size_t)b->num_obs, E = (size_t)b->desc.num_envs;
+    cudaError_t e = cudaMalloc(&b->d_rgb, O * px * 3);
+    if (e == cudaSuccess) e = cudaMalloc(&b->d_depth, O * px * 4);
+    if (e == cudaSuccess) e = cudaMalloc(&b->d_cam_in, O * sizeof(mv_camera));
+    if (e == cudaSuccess && b->desc.max_boxes > 0) {
+        e = cudaMalloc(&b->d_box_in, E * b->desc.max_boxes * sizeof(mv_box));
+        if (e == cudaSuccess) e = cudaMalloc(&b->d_count_in, E * sizeof(int32_t));
+    }
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&b->copy_stream, cudaStreamNonBlocking);
+    for (auto &ev : b->ev_chunk)
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&b->ev_done, cudaEventDisableTiming);
+    if (e != cudaSuccess) {
+        free_host_step(b);
+        cudaGetLastError();
+        return cuda_fail(b, e);
+    }
+    b->host_ready = true;
+    return MV_OK;
+}
+
+// End of a synchronous host step: wait for the stream, then report a staging wait that ran out
+// (the frames of such a step are not valid).
+int finish_host_step(mv_batch *b, cudaStream_t s) {
+    uint32_t word = 0;
+    MV_CUDA(b, cudaMemcpyAsync(&word, b->d_status, 4, cudaMemcpyDeviceToHost, s));
+    MV_CUDA(b, cudaStreamSynchronize(s));
+    return (word & kFlagTimeout) ? MV_ERR_DEVICE_TIMEOUT : MV_OK;
 }
 
 }  // namespace
@@ -228,12 +301,7 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
     b->tiles_x = d.width / 8;
     b->tiles_y = d.height / 4;
     b->mask_words = d.max_boxes > 0 ? (d.max_boxes + 31) / 32 : 1;
-    b->smem_mask_off = round_up(L.block_bytes, 16);
-    b->smem_rel_off = b->smem_mask_off + round_up((uint32_t)(b->tiles_x * b->tiles_y * b->mask_words * 4), 16);
-    b->smem_misc_off = b->smem_rel_off + (uint32_t)(d.max_boxes > 0 ? d.max_boxes : 1) * 32;
-    b->smem_ov_off = b->smem_misc_off + 16 + 6 * 16;   // barrier word, then the 6-entry DDA start table
-    b->smem_bytes = b->smem_ov_off + (uint32_t)(d.max_overlay_rects > 0 ? d.max_overlay_rects : 1) * 32 +
-                    round_up((uint32_t)((b->tiles_x * b->tiles_y + 31) / 32) * 4, 16);
+    b->smem = smem_layout(b, 1);
 
     // kr = tan(hfov/2)/W, ku = (tan(hfov/2)*H/W)/H in double (scalar set-up for the camera kernel)
     const double tx = std::tan((double)d.hfov_rad / 2.0);
@@ -247,22 +315,46 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
     if (e != cudaSuccess || d.device >= ndev) { delete b; return e != cudaSuccess ? MV_ERR_CUDA : MV_ERR_INVALID_ARG; }
     DeviceGuard g(d.device);
     if (!g.ok) { delete b; return MV_ERR_CUDA; }
-    int smem_max = 0;
+    int smem_max = 0, sms = 0;
     e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, d.device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, d.device);
     if (e != cudaSuccess) { delete b; return MV_ERR_CUDA; }
+    b->smem_max = smem_max;
     // the occupancy normally rides in shared memory with the rest of the env block; a grid too large
     // for that keeps it in global memory and stages only the block's tail
-    b->occ_fits_shared = (int)b->smem_bytes <= smem_max;
+    b->occ_fits_shared = (int)b->smem.bytes <= smem_max;
     b->occ_shared = b->occ_fits_shared;
-    if ((int)(b->smem_bytes - L.occ_bytes) > smem_max) { delete b; return MV_ERR_UNSUPPORTED; }
-    e = cudaSuccess;
-    if (b->occ_fits_shared)
-        e = cudaFuncSetAttribute(render_kernel<kRenderThreads, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)b->smem_bytes);
+    if ((int)(b->smem.bytes - L.occ_bytes) > smem_max) { delete b; return MV_ERR_UNSUPPORTED; }
+    // The dynamic shared-memory cap is a property of the kernel function on this device, shared by
+    // every batch: raise it to the device's maximum once, never to one batch's own size.
+    e = cudaFuncSetAttribute(render_kernel<kRenderThreads, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(render_kernel<kRenderThreads, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(b->smem_bytes - L.occ_bytes));
+                                 smem_max);
     if (e != cudaSuccess) { delete b; return MV_ERR_CUDA; }
+    // One CTA per environment (block staged once for all its agents) when that still fills the GPU;
+    // otherwise one CTA per observation.  Cost model: waves of resident CTAs x (agents + fixed part).
+    if (d.agents_per_env > 1) {
+        const mv_batch::Smem all = smem_layout(b, d.agents_per_env);
+        const uint32_t unstaged = b->occ_shared ? 0u : L.occ_bytes;   // never give up staged occupancy for it
+        if ((int)(all.bytes - unstaged) <= smem_max) {
+            auto waves_cost = [&](const mv_batch::Smem &m, int apc) {
+                int per_sm = 0;
+                cudaError_t q = b->occ_shared
+                    ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, render_kernel<kRenderThreads, true>,
+                                                                    kRenderThreads, m.bytes)
+                    : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, render_kernel<kRenderThreads, false>,
+                                                                    kRenderThreads, m.bytes - L.occ_bytes);
+                if (q != cudaSuccess || per_sm < 1) return 1e30;
+                const double slots = (double)per_sm * sms, ctas = (double)b->num_obs / apc;
+                return std::ceil(ctas / slots) * (apc + kCtaFixedCost);
+            };
+            if (waves_cost(all, d.agents_per_env) < waves_cost(b->smem, 1)) {
+                b->smem = all;
+                b->agents_per_cta = b->auto_agents_per_cta = d.agents_per_env;
+            }
+        }
+    }
 
     const size_t blocks_bytes = (size_t)d.num_envs * L.stride;
     bool ok = cudaMalloc(&b->d_env_blocks, blocks_bytes) == cudaSuccess &&
@@ -421,17 +513,9 @@ int mv_step_host(mv_batch *b, const mv_camera *h_cams, const mv_box *h_boxes, co
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const size_t px = (size_t)b->desc.width * b->desc.height;
     const int E = b->desc.num_envs, O = b->num_obs;
-    if (!b->d_rgb) {
-        MV_CUDA(b, cudaMalloc(&b->d_rgb, (size_t)O * px * 3));
-        MV_CUDA(b, cudaMalloc(&b->d_depth, (size_t)O * px * 4));
-        MV_CUDA(b, cudaMalloc(&b->d_cam_in, (size_t)O * sizeof(mv_camera)));
-        if (b->desc.max_boxes > 0) {
-            MV_CUDA(b, cudaMalloc(&b->d_box_in, (size_t)E * b->desc.max_boxes * sizeof(mv_box)));
-            MV_CUDA(b, cudaMalloc(&b->d_count_in, (size_t)E * sizeof(int32_t)));
-        }
-        MV_CUDA(b, cudaStreamCreateWithFlags(&b->copy_stream, cudaStreamNonBlocking));
-        for (auto &ev : b->ev_chunk) MV_CUDA(b, cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
-        MV_CUDA(b, cudaEventCreateWithFlags(&b->ev_done, cudaEventDisableTiming));
+    if (!b->host_ready) {
+        int r = alloc_host_step(b);
+        if (r != MV_OK) return r;
     }
     MV_CUDA(b, cudaMemcpyAsync(b->d_cam_in, h_cams, (size_t)O * sizeof(mv_camera), cudaMemcpyHostToDevice, s));
     if (h_boxes) {
@@ -444,9 +528,11 @@ int mv_step_host(mv_batch *b, const mv_camera *h_cams, const mv_box *h_boxes, co
     int r = launch_cameras(b, b->d_cam_in, s);
     if (r != MV_OK) return r;
     // render chunk by chunk; each chunk's frames start their trip to the host while the next renders
-    const int chunks = O < kHostChunks ? 1 : kHostChunks;
+    // (chunks are whole environments, as the render launch wants when one CTA renders an env)
+    const int A = b->desc.agents_per_env;
+    const int chunks = E < kHostChunks ? 1 : kHostChunks;
     for (int c = 0; c < chunks; ++c) {
-        const int o0 = (int)((int64_t)O * c / chunks), o1 = (int)((int64_t)O * (c + 1) / chunks);
+        const int o0 = (int)((int64_t)E * c / chunks) * A, o1 = (int)((int64_t)E * (c + 1) / chunks) * A;
         r = launch_render(b, b->d_rgb, b->d_depth, o0, o1 - o0, s);
         if (r != MV_OK) return r;
         MV_CUDA(b, cudaEventRecord(b->ev_chunk[c], s));
@@ -458,8 +544,7 @@ int mv_step_host(mv_batch *b, const mv_camera *h_cams, const mv_box *h_boxes, co
     }
     MV_CUDA(b, cudaEventRecord(b->ev_done, b->copy_stream));
     MV_CUDA(b, cudaStreamWaitEvent(s, b->ev_done, 0));
-    MV_CUDA(b, cudaStreamSynchronize(s));
-    return MV_OK;
+    return finish_host_step(b, s);
 }
 
 int mv_step_host_static(mv_batch *b, const mv_camera *h_cams, uint8_t *h_rgb, float *h_depth,
@@ -491,8 +576,7 @@ int mv_step_host_static(mv_batch *b, const mv_camera *h_cams, uint8_t *h_rgb, fl
     if (r != MV_OK) return r;
     MV_CUDA(b, cudaMemcpyAsync(h_rgb, d_rgb, O * px * 3, cudaMemcpyDeviceToHost, s));
     MV_CUDA(b, cudaMemcpyAsync(h_depth, d_depth, O * px * 4, cudaMemcpyDeviceToHost, s));
-    MV_CUDA(b, cudaStreamSynchronize(s));
-    return MV_OK;
+    return finish_host_step(b, s);
 }
 
 int mv_query_status(mv_batch *b, int clear, void *cuda_stream) {
@@ -517,6 +601,20 @@ int mv_debug_occupancy_in_global(mv_batch *b, int on) {
     return MV_OK;
 }
 
+int mv_debug_agents_per_cta(mv_batch *b, int agents_per_cta) {
+    if (!b) return MV_ERR_INVALID_ARG;
+    const int A = b->desc.agents_per_env;
+    int apc = agents_per_cta == 0 ? b->auto_agents_per_cta : agents_per_cta;
+    if (apc != 1 && apc != A) return MV_ERR_INVALID_ARG;
+    const mv_batch::Smem m = smem_layout(b, apc);
+    if ((int)(m.bytes - b->lay.occ_bytes) > b->smem_max) return MV_ERR_UNSUPPORTED;
+    b->occ_fits_shared = (int)m.bytes <= b->smem_max;
+    if (!b->occ_fits_shared) b->occ_shared = false;
+    b->smem = m;
+    b->agents_per_cta = apc;
+    return MV_OK;
+}
+
 int mv_debug_staging(mv_batch *b, int skip_staging, int wait_polls) {
     if (!b || wait_polls < 1 || wait_polls > (1 << 24)) return MV_ERR_INVALID_ARG;
     b->skip_staging = skip_staging ? 1 : 0;
@@ -533,11 +631,7 @@ int mv_destroy(mv_batch *b) {
             if (cudaDeviceSynchronize() != cudaSuccess) rc = MV_ERR_CUDA;
             cudaFree(b->d_env_blocks); cudaFree(b->d_mat); cudaFree(b->d_cams); cudaFree(b->d_status);
             cudaFree(b->d_overlay); cudaFree(b->d_overlay_count); cudaFree(b->d_covered);
-            cudaFree(b->d_rgb); cudaFree(b->d_depth); cudaFree(b->d_cam_in); cudaFree(b->d_box_in);
-            cudaFree(b->d_count_in);
-            if (b->copy_stream) cudaStreamDestroy(b->copy_stream);
-            for (auto &ev : b->ev_chunk) if (ev) cudaEventDestroy(ev);
-            if (b->ev_done) cudaEventDestroy(b->ev_done);
+            free_host_step(b);
             cudaGetLastError();
         }
     }

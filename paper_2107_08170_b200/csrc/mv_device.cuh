@@ -50,8 +50,13 @@ struct RenderParams {
     int W, H, tiles_x, tiles_y, mask_words;
     uint32_t sky_rgbx;
     float miss_depth;
-    uint32_t smem_mask_off, smem_rel_off, smem_misc_off;   // offsets after the env block
-    uint32_t smem_ov_off;              // overlay rectangles of the observation
+    int agents_per_cta;                // observations one CTA renders: 1, or all agents of its env
+    int max_steps;                     // bound of the traversal loop: grid_x + grid_y + grid_z + 3
+    float exit_scale;                  // 1 - (bound on the rounding drift of accumulated crossing times)
+    // shared-memory offsets after the staged env block: tile table, per-agent box masks, per-agent
+    // eye-relative boxes, per-agent camera records + DDA start tables, barrier and flag words,
+    // per-agent overlay rectangles + touched-tile bits
+    uint32_t smem_tile_off, smem_mask_off, smem_rel_off, smem_agent_off, smem_misc_off, smem_ov_off;
     const int4 *overlay;               // [O][max_overlay] 16-byte records, or null
     const int32_t *overlay_count;      // [O]
     int max_overlay;

@@ -446,3 +446,62 @@ def test_fuzz_cameras_anywhere_with_boxes(oracle):
     assert status == 0
     parity.assert_parity(st, "fuzz")
     assert st["pixels"] == E * A * W * H and (g_depth > 0).mean() > 0.2
+
+
+def test_cta_per_environment_equals_cta_per_observation():
+    """The render kernel may give one CTA a whole environment (block staged once for all its agents)
+    or a single observation; both shapes must write the same bytes, overlay and bad cameras included."""
+    from gpu_util import upload_scene
+    B = _binding()
+    cfg = scenes.config("rooms_boxes", num_envs=5)
+    sc = scenes.make_scene(cfg)
+    batch = B.Batch(B.desc_from_config(cfg, 0, max_overlay_rects=2))
+    upload_scene(batch, sc)
+    cams = sc["cams"].clone()
+    cams[7, 3] = torch.tensor([float("nan")]).view(torch.int32)              # one bad camera in the middle of an env
+    d_cams = cams.cuda().contiguous()
+    rects = torch.zeros(cfg.num_obs, 2, 4, dtype=torch.int32)
+    rects[:, 0, 0] = 4 | (2 << 16); rects[:, 0, 1] = 100 | (6 << 16); rects[:, 0, 2] = 0x20C0FF
+    rects[:, 1, 0] = 60 | (40 << 16); rects[:, 1, 1] = 90 | (71 << 16); rects[:, 1, 2] = 0x00FF00
+    count = (torch.arange(cfg.num_obs, dtype=torch.int32) % 3)
+    batch.set_overlays(rects.cuda(), count.cuda())
+    out = {}
+    for apc in (1, cfg.agents):
+        batch.debug_agents_per_cta(apc)
+        batch.set_cameras(d_cams)                                            # (sets the bad-camera flag again)
+        rgb, depth = batch.alloc_outputs()
+        rgb.fill_(9); depth.fill_(-3.0)
+        batch.render_batch(rgb, depth)
+        assert batch.query_status(clear=True) == B.FLAG_BAD_CAMERA
+        out[apc] = (rgb.cpu(), depth.cpu())
+    assert torch.equal(out[1][0], out[cfg.agents][0]) and torch.equal(out[1][1], out[cfg.agents][1])
+    assert (out[1][0][7] == torch.tensor([127, 178, 229], dtype=torch.uint8)).all()
+    with pytest.raises(B.MvError):
+        batch.debug_agents_per_cta(3)
+    batch.debug_agents_per_cta(0)
+    batch.destroy()
+
+
+def test_two_batches_of_different_shape_alive_together():
+    """The kernel's shared-memory cap is per function and device, not per batch: a small batch created
+    after a large one must not make the large one's launch fail."""
+    from gpu_util import upload_scene
+    B = _binding()
+    big_cfg = scenes.config("headline", num_envs=3)
+    small_cfg = scenes.config("tiny")
+    big_sc, small_sc = scenes.make_scene(big_cfg), scenes.make_scene(small_cfg)
+    big = B.Batch(B.desc_from_config(big_cfg))
+    upload_scene(big, big_sc)
+    big.set_cameras(big_sc["cams"].cuda())
+    small = B.Batch(B.desc_from_config(small_cfg))
+    upload_scene(small, small_sc)
+    small.set_cameras(small_sc["cams"].cuda())
+    frames = []
+    for b in (big, small, big):
+        rgb, depth = b.alloc_outputs()
+        b.render_batch(rgb, depth)
+        assert b.query_status() == 0
+        frames.append((rgb.cpu(), depth.cpu()))
+    assert torch.equal(frames[0][0], frames[2][0]) and torch.equal(frames[0][1], frames[2][1])
+    assert (frames[0][1] > 0).any() and (frames[1][1] > 0).any()
+    big.destroy(); small.destroy()

@@ -347,3 +347,61 @@ def test_tie_breaks_voxel_before_box_and_lower_box_first(oracle):
     rgb, depth, ids = oracle.render_obs(d, np.zeros_like(grid), boxes, 2, pal, cam)
     assert (ids[:, c, 0] == 1).all() and (ids[:, c, 1] == 0).all()                 # lower box index wins
     assert (rgb[:, c, 1] > 0).all() and (rgb[:, c, 2] == 0).all()                  # box 0's colour (green)
+
+
+def test_axis_parallel_rays_zero_direction_component(oracle):
+    """Rays with a direction component that is EXACTLY zero (an odd image size puts a pixel centre on
+    the view axis: a = 2px+1-W = 0 in the centre column, b = H-1-2py = 0 in the centre row, and with
+    yaw = pitch = 0 the basis has exact zeros).  Along such an axis the ray never moves, so a slab is
+    crossed iff the eye lies within it, both ends included: geometry fixes every value below."""
+    W = H = 5
+    gx, gy, gz = 8, 16, 12
+    grid = np.zeros((gy, gz, gx), np.uint8)
+    grid[:, 9, :] = 1                                          # wall plane k = 9
+    pal = PALETTE_1
+    cx, cy, cz = 3.0, 7.5, 1.25                                # cx sits exactly on a cell face (x = 3)
+    # boxes in front of the wall, all spanning y 7..8 unless said otherwise; material 1
+    boxes = box_rows([
+        ((2.5, 7.0, 4.0), (3.5, 8.0, 4.5), 1),                 # 0: x-range contains cx        -> centre column hits it
+        ((3.0, 7.0, 5.0), (3.5, 8.0, 5.5), 1),                 # 1: cx exactly on lo.x         -> counts as inside
+        ((2.5, 7.0, 6.0), (3.0, 8.0, 6.5), 1),                 # 2: cx exactly on hi.x         -> counts as inside
+        ((3.25, 7.0, 3.0), (3.75, 8.0, 3.5), 1),               # 3: x-range excludes cx (nearest of all) -> missed
+        ((2.0, 7.75, 2.0), (4.0, 8.0, 2.5), 1),                # 4: y-range excludes cy (nearer still)    -> missed by the centre row
+    ])
+    d = _desc(oracle, grid, W, H, max_boxes=8)
+    cam = cam_row(cx, cy, cz, 0.0, 0.0)
+
+    def centre(nboxes, which):
+        rgb, depth, ids = oracle.render_obs(d, grid, boxes[which] if nboxes else None, nboxes, pal, cam)
+        return rgb, depth, ids
+
+    # no boxes: the centre pixel looks straight down +z (d = (0, 0, 1)) and meets the wall at k - cz
+    rgb, depth, ids = centre(0, slice(0, 0))
+    assert ids[2, 2].tolist()[0] == 0 and ids[2, 2, 2] == 4    # a voxel, its -z face
+    assert abs(depth[2, 2] - (9 - cz)) <= 1e-6
+    # cx = 3.0 lies on the shared face of x cells 2 and 3: both closed slabs contain it, the lowest index wins
+    assert ids[2, 2, 1] == 2 + gx * (9 + gz * 7)
+    # the whole centre column has d_x == 0 and the whole centre row d_y == 0: the wall voxels they meet
+    # lie in the eye's own x column / y layer
+    for py in range(H):
+        assert ids[py, 2, 0] == 0 and ids[py, 2, 1] % gx in (2, 3)
+    for px in range(W):
+        assert ids[2, px, 0] == 0 and (ids[2, px, 1] // (gx * gz)) == 7
+
+    want = {0: 4.0 - cz, 1: 5.0 - cz, 2: 6.0 - cz}
+    for b, t in want.items():                                  # each containing box alone is hit head-on at its near z face
+        rgb, depth, ids = centre(1, slice(b, b + 1))
+        assert ids[2, 2].tolist() == [1, 0, 4], (b, ids[2, 2])
+        assert abs(depth[2, 2] - t) <= 1e-6
+    for b in (3, 4):                                           # boxes that exclude the eye's coordinate are missed
+        rgb, depth, ids = centre(1, slice(b, b + 1))
+        assert ids[2, 2, 0] == 0 and abs(depth[2, 2] - (9 - cz)) <= 1e-6, b
+    # all together: box 4 and box 3 are nearer but missed; box 0 is the nearest that is hit
+    rgb, depth, ids = centre(5, slice(0, 5))
+    assert ids[2, 2].tolist() == [1, 0, 4] and abs(depth[2, 2] - (4.0 - cz)) <= 1e-6
+    # box 4 is missed by the centre row only.  The row above looks up with d_y = b*ty/H = 2*1/5 = 0.4; at the
+    # box's near z face (t = 2.0 - cz = 0.75) it is at y = 7.5 + 0.3 = 7.8, inside [7.75, 8]: a hit on the
+    # -z face at depth 0.75
+    assert ids[1, 2].tolist() == [1, 4, 4] and abs(depth[1, 2] - 0.75) <= 1e-6
+    # colours: ambient-only (-z faces): floor(palette * 0.3 + 0.5)
+    assert (rgb[2, 2] == np.floor(np.array(PALETTE_1[1], float) * 0.3 + 0.5)).all()
