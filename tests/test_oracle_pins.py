@@ -359,14 +359,14 @@ def test_axis_parallel_rays_zero_direction_component(oracle):
     grid = np.zeros((gy, gz, gx), np.uint8)
     grid[:, 9, :] = 1                                          # wall plane k = 9
     pal = PALETTE_1
-    cx, cy, cz = 3.0, 7.5, 1.25                                # cx sits exactly on a cell face (x = 3)
+    cx, cy, cz = 4.0, 7.5, 1.25                                # cx sits exactly on a cell face (x = 4)
     # boxes in front of the wall, all spanning y 7..8 unless said otherwise; material 1
     boxes = box_rows([
-        ((2.5, 7.0, 4.0), (3.5, 8.0, 4.5), 1),                 # 0: x-range contains cx        -> centre column hits it
-        ((3.0, 7.0, 5.0), (3.5, 8.0, 5.5), 1),                 # 1: cx exactly on lo.x         -> counts as inside
-        ((2.5, 7.0, 6.0), (3.0, 8.0, 6.5), 1),                 # 2: cx exactly on hi.x         -> counts as inside
-        ((3.25, 7.0, 3.0), (3.75, 8.0, 3.5), 1),               # 3: x-range excludes cx (nearest of all) -> missed
-        ((2.0, 7.75, 2.0), (4.0, 8.0, 2.5), 1),                # 4: y-range excludes cy (nearer still)    -> missed by the centre row
+        ((3.5, 7.0, 4.0), (4.5, 8.0, 4.5), 1),                 # 0: x-range contains cx        -> centre column hits it
+        ((4.0, 7.0, 5.0), (4.5, 8.0, 5.5), 1),                 # 1: cx exactly on lo.x         -> counts as inside
+        ((3.5, 7.0, 6.0), (4.0, 8.0, 6.5), 1),                 # 2: cx exactly on hi.x         -> counts as inside
+        ((4.25, 7.0, 3.0), (4.75, 8.0, 3.5), 1),               # 3: x-range excludes cx (nearest of all) -> missed
+        ((3.0, 7.75, 2.0), (5.0, 8.0, 2.5), 1),                # 4: y-range excludes cy (nearer still)    -> missed by the centre row
     ])
     d = _desc(oracle, grid, W, H, max_boxes=8)
     cam = cam_row(cx, cy, cz, 0.0, 0.0)
@@ -379,13 +379,13 @@ def test_axis_parallel_rays_zero_direction_component(oracle):
     rgb, depth, ids = centre(0, slice(0, 0))
     assert ids[2, 2].tolist()[0] == 0 and ids[2, 2, 2] == 4    # a voxel, its -z face
     assert abs(depth[2, 2] - (9 - cz)) <= 1e-6
-    # cx = 3.0 lies on the shared face of x cells 2 and 3: both closed slabs contain it, the lowest index wins
-    assert ids[2, 2, 1] == 2 + gx * (9 + gz * 7)
+    # cx = 4.0 lies on the shared face of x cells 3 and 4: both closed slabs contain it, the lowest index wins
+    assert ids[2, 2, 1] == 3 + gx * (9 + gz * 7)
     # the whole centre column has d_x == 0 and the whole centre row d_y == 0: the wall voxels they meet
     # lie in the eye's own x column / y layer
     for py in range(H):
-        assert ids[py, 2, 0] == 0 and ids[py, 2, 1] % gx in (2, 3)
-    for px in range(W):
+        assert ids[py, 2, 0] == 0 and ids[py, 2, 1] % gx in (3, 4)
+    for px in (1, 2, 3):                                       # (the outermost two leave the 8-wide grid before the wall)
         assert ids[2, px, 0] == 0 and (ids[2, px, 1] // (gx * gz)) == 7
 
     want = {0: 4.0 - cz, 1: 5.0 - cz, 2: 6.0 - cz}
