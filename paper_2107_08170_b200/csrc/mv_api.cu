@@ -32,6 +32,7 @@ struct mv_batch {
     mv_batch_desc desc;
     int num_obs = 0;
     size_t nvox = 0;
+    size_t mat_bytes_per_env = 0;       // material store: one byte per voxel index (columns padded to 2^ysh)
     EnvLayout lay{};
     unsigned char *d_env_blocks = nullptr;
     uint8_t *d_mat = nullptr;
@@ -291,7 +292,10 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
     b->missing_grid = b->missing_palette = d.num_envs;
 
     EnvLayout &L = b->lay;
-    L.occ_bytes = round_up((uint32_t)(b->nvox / 8), 16);
+    L.ysh = 5;                                              // bits per (x, z) column: a power of two >= grid_y, >= 32
+    while ((1 << L.ysh) < d.grid_y) L.ysh++;
+    L.occ_bytes = (uint32_t)(((size_t)d.grid_x * d.grid_z << L.ysh) / 8);
+    b->mat_bytes_per_env = (size_t)d.grid_x * d.grid_z << L.ysh;
     L.lut_off = L.occ_bytes;
     L.box_off = L.lut_off + round_up(kFaces * d.palette_size * 4, 16);
     L.count_off = L.box_off + (uint32_t)d.max_boxes * 32;
@@ -358,7 +362,7 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
 
     const size_t blocks_bytes = (size_t)d.num_envs * L.stride;
     bool ok = cudaMalloc(&b->d_env_blocks, blocks_bytes) == cudaSuccess &&
-              cudaMalloc(&b->d_mat, (size_t)d.num_envs * b->nvox) == cudaSuccess &&
+              cudaMalloc(&b->d_mat, (size_t)d.num_envs * b->mat_bytes_per_env) == cudaSuccess &&
               cudaMalloc(&b->d_cams, (size_t)b->num_obs * sizeof(CamRec)) == cudaSuccess &&
               cudaMalloc(&b->d_status, 16) == cudaSuccess;
     if (ok && d.max_overlay_rects > 0)
@@ -388,11 +392,12 @@ int mv_upload_worlds(mv_batch *b, int env_begin, int env_count, const uint8_t *d
     if (!g.ok) return MV_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     if (d_grid) {
-        const size_t threads = b->nvox / 32 * (size_t)env_count;
+        const size_t threads = ((size_t)(b->desc.grid_x / 4) * b->desc.grid_z << (b->lay.ysh - 5)) * (size_t)env_count;
         const size_t blocks = (threads + 255) / 256;
         if (blocks > 0x7fffffffull) return MV_ERR_INVALID_ARG;
-        pack_grid_kernel<<<(unsigned)blocks, 256, 0, s>>>(d_grid, b->d_env_blocks, b->d_mat, b->lay, b->nvox,
-                                                           env_begin, env_count, b->desc.palette_size, b->d_status);
+        pack_grid_kernel<<<(unsigned)blocks, 256, 0, s>>>(d_grid, b->d_env_blocks, b->d_mat, b->lay, b->desc.grid_x,
+                                                           b->desc.grid_y, b->desc.grid_z, env_begin, env_count,
+                                                           b->desc.palette_size, b->d_status);
         b->launches++;
         MV_CUDA(b, cudaGetLastError());
         occupied_bounds_kernel<<<env_count, 256, 0, s>>>(b->d_env_blocks, b->lay, env_begin, b->desc.grid_x,
@@ -477,17 +482,22 @@ int mv_merge_voxels(mv_batch *b, int env_begin, int env_count, mv_box *d_boxes_o
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const size_t words = b->nvox / 32;
     if (!b->d_covered) {
-        size_t chunk = kMergeScratchBytes / (words * 4);
+        size_t chunk = kMergeScratchBytes / (words * 4 * 2);       // coverage bits + x-packed occupancy per env
         chunk = chunk < 1 ? 1 : (chunk > (size_t)b->desc.num_envs ? (size_t)b->desc.num_envs : chunk);
-        MV_CUDA(b, cudaMalloc(&b->d_covered, chunk * words * 4));
+        MV_CUDA(b, cudaMalloc(&b->d_covered, chunk * words * 4 * 2));
         b->merge_chunk = (int)chunk;
     }
     const int kMergeChunk = b->merge_chunk;
     for (int e0 = 0; e0 < env_count; e0 += kMergeChunk) {
         const int n = env_count - e0 < kMergeChunk ? env_count - e0 : kMergeChunk;
+        uint32_t *occx = b->d_covered + (size_t)kMergeChunk * words;
         MV_CUDA(b, cudaMemsetAsync(b->d_covered, 0, (size_t)n * words * 4, s));
+        xpack_kernel<<<(unsigned)(((size_t)n * words + 255) / 256), 256, 0, s>>>(
+            b->d_env_blocks, b->lay, env_begin + e0, n, b->desc.grid_x, b->desc.grid_y, b->desc.grid_z, occx);
+        b->launches++;
+        MV_CUDA(b, cudaGetLastError());
         merge_voxels_kernel<<<(n * 32 + 127) / 128, 128, 0, s>>>(
-            b->d_env_blocks, b->d_mat, b->lay, env_begin + e0, n, b->desc.grid_x, b->desc.grid_y, b->desc.grid_z,
+            occx, b->d_mat, b->lay, env_begin + e0, n, b->desc.grid_x, b->desc.grid_y, b->desc.grid_z,
             b->d_covered, reinterpret_cast<uint4 *>(d_boxes_out + (size_t)e0 * max_out), d_count_out + e0, max_out);
         b->launches++;
         MV_CUDA(b, cudaGetLastError());

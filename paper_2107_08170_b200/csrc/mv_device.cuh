@@ -25,19 +25,28 @@ static_assert(sizeof(CamRec) == 64, "CamRec must be 64 bytes");
 
 // One environment's render inputs, contiguous in HBM so that a single bulk copy stages them
 // into shared memory:  [occupancy bits | shade LUT | boxes | box count + occupied bounds].
+// Occupancy is packed along y: the (x, z) column owns 2^ysh consecutive bits (2^ysh >= grid_y, at
+// least 32), bit index u = ((x + grid_x*z) << ysh) | y, bit u&31 of word u>>5.  A walk along x or z
+// therefore moves by whole words and a walk along y stays inside the column's word(s); for grids
+// up to 32 voxels high a column is exactly one word.  The material store uses the same index u.
 struct EnvLayout {
-    uint32_t occ_bytes;     // grid_x*grid_y*grid_z/8 rounded up to 16
+    uint32_t occ_bytes;     // grid_x*grid_z*2^ysh/8
     uint32_t lut_off;       // 7*palette_size RGBX words
     uint32_t box_off;       // max_boxes * 32 bytes
     uint32_t count_off;     // 32 bytes: {box count, lo x,y,z, hi x,y,z, pad}; [lo, hi) = cell box
                             // that contains every filled voxel (lo > hi when the grid is empty)
     uint32_t block_bytes;   // bytes staged per CTA (multiple of 16)
     uint32_t stride;        // distance between envs in HBM (multiple of 128)
+    uint32_t ysh;           // log2 of the bits per (x, z) column
 };
+
+__host__ __device__ __forceinline__ uint32_t voxel_index(uint32_t ysh, int gx, int x, int y, int z) {
+    return ((uint32_t)(x + gx * z) << ysh) | (uint32_t)y;
+}
 
 struct RenderParams {
     const unsigned char *env_blocks;   // [E] EnvLayout blocks
-    const uint8_t *mat;                // [E][nvox] material ids (clamped to palette at upload)
+    const uint8_t *mat;                // [E][grid_x*grid_z << ysh] material ids by voxel index (clamped at upload)
     const CamRec *cams;                // [O]
     uint8_t *rgb;                      // [O][H][W][3]
     float *depth;                      // [O][H][W]

@@ -12,35 +12,59 @@ __device__ __forceinline__ uint32_t nz_bits4(uint32_t v) {
     return (ones * 0x01020408u) >> 24;
 }
 
-// uint8 grid [env][y][z][x] -> 1 bit per voxel (bit v&31 of word v>>5, v = x + gx*(z + gz*y))
-// inside the env block, plus a material copy with ids clamped to the palette.  One thread
-// packs 32 voxels.
+// 4 x 4 byte transpose: in[i] holds byte c of column c at height i; out[c] the four heights of column c.
+__device__ __forceinline__ void transpose4x4(const uint32_t in[4], uint32_t out[4]) {
+    const uint32_t a = __byte_perm(in[0], in[1], 0x5140), b = __byte_perm(in[2], in[3], 0x5140);   // c0h0 c0h1 c1h0 c1h1 | ..h2 h3
+    const uint32_t c = __byte_perm(in[0], in[1], 0x7362), d = __byte_perm(in[2], in[3], 0x7362);   // c2h0 c2h1 c3h0 c3h1 | ..h2 h3
+    out[0] = __byte_perm(a, b, 0x5410); out[1] = __byte_perm(a, b, 0x7632);
+    out[2] = __byte_perm(c, d, 0x5410); out[3] = __byte_perm(c, d, 0x7632);
+}
+
+// uint8 grid [env][y][z][x] -> occupancy bits packed along y inside the env block (see EnvLayout)
+// plus a material copy by voxel index with ids clamped to the palette.  One thread packs 32
+// heights of four neighbouring columns: 32 four-byte loads, four words and 128 material bytes out.
 __global__ void pack_grid_kernel(const uint8_t *__restrict__ grid, unsigned char *__restrict__ env_blocks,
-                                 uint8_t *__restrict__ mat, EnvLayout lay, size_t nvox, int env_begin,
+                                 uint8_t *__restrict__ mat, EnvLayout lay, int gx, int gy, int gz, int env_begin,
                                  int env_count, int palette, uint32_t *status)
 {
-    const size_t words_per_env = nvox / 32;
+    const int xg_n = gx / 4, col_words = 1 << (lay.ysh - 5);
+    const size_t per_env = (size_t)xg_n * gz * col_words;
     const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (gid >= words_per_env * (size_t)env_count) return;
-    const size_t e = gid / words_per_env, w = gid - e * words_per_env;
-    const uint4 *src = reinterpret_cast<const uint4 *>(grid + e * nvox + w * 32);
-    uint4 q[2] = {src[0], src[1]};
-    uint32_t *v = reinterpret_cast<uint32_t *>(q);
+    if (gid >= per_env * (size_t)env_count) return;
+    const size_t e = gid / per_env;
+    size_t r = gid - e * per_env;
+    const int wq = (int)(r / ((size_t)xg_n * gz));
+    r -= (size_t)wq * xg_n * gz;
+    const int z = (int)(r / xg_n), xg = (int)(r - (size_t)z * xg_n);
+    const size_t nvox = (size_t)gx * gy * gz;
+    const uint8_t *src = grid + e * nvox + (size_t)z * gx + 4 * xg;
     const uint32_t cap = (uint32_t)(palette - 1) * 0x01010101u;
-    uint32_t bits = 0, clamped = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const uint32_t orig = v[i];
-        bits |= nz_bits4(orig) << (4 * i);          // filled = id != 0, decided before clamping
-        const uint32_t c = __vminu4(orig, cap);
-        clamped |= c ^ orig;
-        v[i] = c;
-    }
+    uint32_t bits[4] = {0, 0, 0, 0}, clamped = 0;
     const size_t env = (size_t)env_begin + e;
-    reinterpret_cast<uint32_t *>(env_blocks + env * lay.stride)[w] = bits;
-    uint4 *dst = reinterpret_cast<uint4 *>(mat + env * nvox + w * 32);
-    dst[0] = q[0];
-    dst[1] = q[1];
+    const uint32_t u0 = voxel_index(lay.ysh, gx, 4 * xg, 32 * wq, z);
+    uint8_t *mdst = mat + env * ((size_t)gx * gz << lay.ysh) + u0;
+#pragma unroll
+    for (int h0 = 0; h0 < 32; h0 += 4) {
+        uint32_t v[4], t[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int y = 32 * wq + h0 + i;
+            const uint32_t orig = y < gy ? *reinterpret_cast<const uint32_t *>(src + (size_t)y * gz * gx) : 0u;
+            const uint32_t nz = __vcmpne4(orig, 0u);               // 0xff per filled byte, decided before clamping
+#pragma unroll
+            for (int c = 0; c < 4; ++c) bits[c] |= ((nz >> (8 * c)) & 1u) << (h0 + i);
+            const uint32_t cl = __vminu4(orig, cap);
+            clamped |= cl ^ orig;
+            v[i] = cl;
+        }
+        transpose4x4(v, t);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            *reinterpret_cast<uint32_t *>(mdst + ((size_t)c << lay.ysh) + h0) = t[c];
+    }
+    uint32_t *occ = reinterpret_cast<uint32_t *>(env_blocks + env * lay.stride);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) occ[(u0 >> 5) + ((uint32_t)c << (lay.ysh - 5))] = bits[c];
     if (clamped) atomicOr(status, kFlagMaterial);
 }
 
@@ -51,27 +75,17 @@ __global__ void occupied_bounds_kernel(unsigned char *__restrict__ env_blocks, E
 {
     unsigned char *blk = env_blocks + (size_t)(env_begin + blockIdx.x) * lay.stride;
     const uint32_t *occ = reinterpret_cast<const uint32_t *>(blk);
-    const int nwords = gx * gy * gz / 32;
+    const int wsh = lay.ysh - 5;                   // log2 of the words per column
+    const int nwords = (gx * gz) << wsh;
     int lo[3] = {gx, gy, gz}, hi[3] = {-1, -1, -1};
-    const bool row_aligned = (gx % 32) == 0;       // then a 32-voxel word lies inside one x-row
     for (int w = threadIdx.x; w < nwords; w += blockDim.x) {
-        uint32_t m = occ[w];
+        const uint32_t m = occ[w];
         if (!m) continue;
-        if (row_aligned) {
-            const int v = w * 32, x = v % gx, r = v / gx, z = r % gz, y = r / gz;
-            lo[0] = min(lo[0], x + __ffs(m) - 1); hi[0] = max(hi[0], x + 31 - __clz(m));
-            lo[1] = min(lo[1], y); hi[1] = max(hi[1], y);
-            lo[2] = min(lo[2], z); hi[2] = max(hi[2], z);
-            continue;
-        }
-        while (m) {
-            const int v = w * 32 + (__ffs(m) - 1);
-            m &= m - 1;
-            const int x = v % gx, r = v / gx, z = r % gz, y = r / gz;
-            lo[0] = min(lo[0], x); hi[0] = max(hi[0], x);
-            lo[1] = min(lo[1], y); hi[1] = max(hi[1], y);
-            lo[2] = min(lo[2], z); hi[2] = max(hi[2], z);
-        }
+        const int col = w >> wsh, y0 = (w - (col << wsh)) * 32;
+        const int x = col % gx, z = col / gx;
+        lo[0] = min(lo[0], x); hi[0] = max(hi[0], x);
+        lo[1] = min(lo[1], y0 + __ffs(m) - 1); hi[1] = max(hi[1], y0 + 31 - __clz(m));
+        lo[2] = min(lo[2], z); hi[2] = max(hi[2], z);
     }
     __shared__ int s_lo[3], s_hi[3];
     if (threadIdx.x < 3) { s_lo[threadIdx.x] = 1 << 30; s_hi[threadIdx.x] = -1; }
@@ -178,8 +192,8 @@ __global__ void camera_kernel(const int32_t *__restrict__ cams, CamRec *__restri
 
 // True iff the body box around (x, y, z) lies inside the grid and touches no filled voxel
 // (cells floor(lo)..floor(hi) on every axis, ends included).
-__device__ __forceinline__ bool body_free(const uint32_t *occ, int gx, int gy, int gz, float x, float y, float z,
-                                          float hw, float below, float above)
+__device__ __forceinline__ bool body_free(const uint32_t *occ, uint32_t ysh, int gx, int gy, int gz, float x, float y,
+                                          float z, float hw, float below, float above)
 {
     const float lx = __fsub_rn(x, hw), hx = __fadd_rn(x, hw);
     const float ly = __fsub_rn(y, below), hy = __fadd_rn(y, above);
@@ -192,7 +206,7 @@ __device__ __forceinline__ bool body_free(const uint32_t *occ, int gx, int gy, i
     for (int j = j0; j <= j1; ++j)
         for (int k = k0; k <= k1; ++k)
             for (int i = i0; i <= i1; ++i) {
-                const int v = i + gx * (k + gz * j);
+                const uint32_t v = voxel_index(ysh, gx, i, j, k);
                 if ((occ[v >> 5] >> (v & 31)) & 1u) return false;
             }
     return true;
@@ -224,8 +238,8 @@ __global__ void move_agents_kernel(int32_t *__restrict__ cams, const float4 *__r
     unsigned char *blk = env_blocks + (size_t)(o / agents) * lay.stride;
     const uint32_t *occ = reinterpret_cast<const uint32_t *>(blk);
     float nx = x, nz = z;
-    if (body_free(occ, gx, gy, gz, x_try, y, nz, hw, below, above)) nx = x_try;
-    if (body_free(occ, gx, gy, gz, nx, y, z_try, hw, below, above)) nz = z_try;
+    if (body_free(occ, lay.ysh, gx, gy, gz, x_try, y, nz, hw, below, above)) nx = x_try;
+    if (body_free(occ, lay.ysh, gx, gy, gz, nx, y, z_try, hw, below, above)) nz = z_try;
     c[0] = __float_as_int(nx); c[2] = __float_as_int(nz);
     c[3] = __float_as_int(yaw); c[4] = __float_as_int(pitch);
     const int self_box = c[5];
@@ -238,13 +252,34 @@ __global__ void move_agents_kernel(int32_t *__restrict__ cams, const float4 *__r
     }
 }
 
+// Occupancy of the envs of one merge launch re-packed along x (bit v&31 of word v>>5, v = x + gx*(z + gz*y)),
+// the order in which the merge sweeps.  One thread per output word; scratch, off the per-step path.
+__global__ void xpack_kernel(const unsigned char *__restrict__ env_blocks, EnvLayout lay, int env_begin, int env_count,
+                             int gx, int gy, int gz, uint32_t *__restrict__ out)
+{
+    const size_t nwords = (size_t)gx * gy * gz / 32;
+    const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (gid >= nwords * (size_t)env_count) return;
+    const size_t e = gid / nwords, w = gid - e * nwords;
+    const uint32_t *occ = reinterpret_cast<const uint32_t *>(env_blocks + (size_t)(env_begin + e) * lay.stride);
+    uint32_t word = 0;
+    for (int b = 0; b < 32; ++b) {
+        const size_t v = w * 32 + b;
+        const int x = (int)(v % gx), r = (int)(v / gx), z = r % gz, y = r / gz;
+        const uint32_t u = voxel_index(lay.ysh, gx, x, y, z);
+        word |= ((occ[u >> 5] >> (u & 31)) & 1u) << b;
+    }
+    out[gid] = word;
+}
+
 // Greedy merging of an env's voxels into boxes (paper Section 3.3), one warp per env, in the
 // same order as a serial sweep: the warp finds the first filled, uncovered voxel in index order,
 // grows a box along +x, then +z, then +y while every cell of the new row / slab is filled,
-// uncovered and of the same material, emits it and marks it covered.  `covered` is scratch:
-// one bit per voxel per env of this launch, zeroed by the caller; it is read around L1 (ld.cg)
-// because lanes read bits that other lanes set with atomics.
-__global__ void merge_voxels_kernel(const unsigned char *__restrict__ env_blocks, const uint8_t *__restrict__ mat,
+// uncovered and of the same material, emits it and marks it covered.  `occx` is the x-packed copy
+// of the occupancy made by xpack_kernel; `covered` is scratch in the same packing, one bit per
+// voxel per env of this launch, zeroed by the caller; it is read around L1 (ld.cg) because lanes
+// read bits that other lanes set with atomics.
+__global__ void merge_voxels_kernel(const uint32_t *__restrict__ occx, const uint8_t *__restrict__ mat,
                                     EnvLayout lay, int env_begin, int env_count, int gx, int gy, int gz,
                                     uint32_t *__restrict__ covered, uint4 *__restrict__ boxes_out,
                                     int32_t *__restrict__ count_out, int max_out)
@@ -254,15 +289,15 @@ __global__ void merge_voxels_kernel(const unsigned char *__restrict__ env_blocks
     if (e >= env_count) return;
     const size_t nvox = (size_t)gx * gy * gz;
     const int nwords = (int)(nvox / 32);
-    const uint32_t *occ = reinterpret_cast<const uint32_t *>(env_blocks + (size_t)(env_begin + e) * lay.stride);
-    const uint8_t *m_env = mat + (size_t)(env_begin + e) * nvox;
+    const uint32_t *occ = occx + (size_t)e * nwords;
+    const uint8_t *m_env = mat + (size_t)(env_begin + e) * ((size_t)gx * gz << lay.ysh);
     uint32_t *cov = covered + (size_t)e * nwords;
     uint4 *out = boxes_out + (size_t)e * max_out * 2;
     const unsigned full = 0xffffffffu;
     auto open = [&](int i, int j, int k, int m) -> bool {
         const int v = i + gx * (k + gz * j);
         const uint32_t bit = 1u << (v & 31);
-        return (occ[v >> 5] & bit) && !(__ldcg(&cov[v >> 5]) & bit) && m_env[v] == m;
+        return (occ[v >> 5] & bit) && !(__ldcg(&cov[v >> 5]) & bit) && m_env[voxel_index(lay.ysh, gx, i, j, k)] == m;
     };
     int count = 0;
     for (int w0 = 0; w0 < nwords; w0 += 32) {
@@ -277,7 +312,7 @@ __global__ void merge_voxels_kernel(const unsigned char *__restrict__ env_blocks
             const uint32_t word = __shfl_sync(full, mine, src);
             const int v = (w0 + src) * 32 + (__ffs(word) - 1);
             const int i = v % gx, r = v / gx, k = r % gz, j = r / gz;
-            const int m = m_env[v];
+            const int m = m_env[voxel_index(lay.ysh, gx, i, j, k)];
             int w = 1, d = 1, h = 1;
             for (;;) {                                           // +x, 32 cells per vote
                 const int a = w + lane;

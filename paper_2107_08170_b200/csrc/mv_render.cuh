@@ -85,7 +85,8 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
 // z) advances: crossing time += dt, voxel index += stride; then the new cell's occupancy bit is
 // tested.  Two registers alternate as t, so that after a hit the time at which the filled cell was
 // entered is still there.  The voxel index carries 8x the shared-memory byte address of the occupancy
-// grid, so (index >> 3) & ~3 is the word's address and index & 31 the bit.
+// grid, so (index >> 3) & ~3 is the word's address and index & 31 the bit (the index is
+// ((x + grid_x*z) << ysh) | y: steps along x and z change the word, steps along y the bit).
 #if defined(MV_PROBE) && MV_PROBE == 9
 #define MV_DDA_COUNT " add.f32 ns, ns, 0f3F800000;\n"
 #define MV_DDA_COUNT_OUT " mov.f32 %1, ns;\n"
@@ -263,7 +264,8 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
 
     // ---- per-agent traversal set-up and box binning
     const int gx = p.gx, gz = p.gz;
-    const int stride_z = gx, stride_y = gx * gz;
+    // voxel-index strides of the y-packed layout: x and z move by whole columns, y by single bits
+    const int stride_x = 1 << p.lay.ysh, stride_z = gx << p.lay.ysh, stride_y = 1;
     // Traversal is confined to the cell box [lo, hi) that holds every filled voxel of this env
     // (nothing outside it can be hit), so rays that leave it, e.g. into the sky, stop there.
     const int lox = s_count[1], loy = s_count[2], loz = s_count[3];
@@ -287,13 +289,13 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         if (cam_in) { cx0 = (int)floorf(c0.x); cy0 = (int)floorf(c0.y); cz0 = (int)floorf(c0.z); }
         const int cc = ax == 0 ? cx0 : (ax == 1 ? cy0 : cz0);
         const int lo_c = ax == 0 ? lox : (ax == 1 ? loy : loz), hi_c = ax == 0 ? hix : (ax == 1 ? hiy : hiz);
-        const int st = ax == 0 ? 1 : (ax == 1 ? stride_y : stride_z);
+        const int st = ax == 0 ? stride_x : (ax == 1 ? stride_y : stride_z);
         s_dda[kDdaVecs * ag + e] = make_float4(neg ? (float)cc - Pc : (float)(cc + 1) - Pc,
                                                neg ? (float)(cc - lo_c) : (float)(hi_c - 1 - cc),
                                                __int_as_float(neg ? -st : st),
                                                __uint_as_float(lut_base + (uint32_t)((2 * ax + neg) * P_ * 4)));
         if (e == 0) {
-            const int vi0 = cx0 + stride_z * cz0 + stride_y * cy0;
+            const int vi0 = stride_x * cx0 + stride_z * cz0 + stride_y * cy0;
             const bool filled = cam_in && ((s_occ[vi0 >> 5] >> (vi0 & 31)) & 1u);
             float4 *slot = &s_agent[kAgentRecVecs * ag + 3];
             slot->x = __uint_as_float((uint32_t)vi0 + vi_bias);
@@ -350,7 +352,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     }
     __syncthreads();
 
-    const uint8_t *mat_env = p.mat + (size_t)env * ((size_t)gx * p.gy * gz) - vi_bias;
+    const uint8_t *mat_env = p.mat + (size_t)env * ((size_t)gx * gz << p.lay.ysh) - vi_bias;
     const float flox = (float)lox, floy = (float)loy, floz = (float)loz;
     const float fhix = (float)hix, fhiy = (float)hiy, fhiz = (float)hiz;
 
@@ -477,7 +479,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                 if (eaxis == 1) cy = ngy ? hiy - 1 : loy;
                 if (eaxis == 2) cz = ngz ? hiz - 1 : loz;
                 if (!alive) { cx = cy = cz = 0; }
-                const int v = cx + stride_z * cz + stride_y * cy;
+                const int v = stride_x * cx + stride_z * cz + stride_y * cy;
                 vi = (uint32_t)v + vi_bias;
                 t0x = ((float)(cx + (ngx ? 0 : 1)) - Px) * ix;
                 t0y = ((float)(cy + (ngy ? 0 : 1)) - Py) * iy;
