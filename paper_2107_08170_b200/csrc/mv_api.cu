@@ -48,7 +48,7 @@ struct mv_batch {
     bool has_cams = false;
     double kr = 0, ku = 0;
     uint32_t sky_rgbx = 0;
-    struct Smem { uint32_t tile_off, mask_off, rel_off, agent_off, misc_off, ov_off, bytes; };
+    struct Smem { uint32_t tile_off, agent_off, agent_stride, agent_ov_off, agent_mask_off, agent_ovtile_off, misc_off, bytes; };
     Smem smem{};                        // shared-memory layout of the render kernel for agents_per_cta
     int agents_per_cta = 1;             // observations one CTA renders: 1, or every agent of its env
     int tiles_x = 0, tiles_y = 0, mask_words = 0;
@@ -98,21 +98,30 @@ struct DeviceGuard {
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Shared-memory layout of the render kernel when one CTA renders `apc` observations of an env:
-// staged env block, tile table, then per-agent box masks, eye-relative boxes, camera records and
-// DDA start tables, the barrier and flag words, and per-agent overlay rectangles + touched-tile bits.
+// staged env block, tile table, then one block per agent (camera record and DDA start table,
+// eye-relative boxes, overlay rectangles, per-tile box masks, per-tile overlay bits), then the
+// barrier and flag words.
 mv_batch::Smem smem_layout(const mv_batch *b, int apc) {
     const mv_batch_desc &d = b->desc;
-    const uint32_t ntiles = (uint32_t)(b->tiles_x * b->tiles_y), a = (uint32_t)apc;
+    const uint32_t ntiles = (uint32_t)(b->tiles_x * b->tiles_y);
     mv_batch::Smem m{};
     m.tile_off = round_up(b->lay.block_bytes, 16);
-    m.mask_off = m.tile_off + ntiles * 16;
-    m.rel_off = m.mask_off + round_up(a * ntiles * (uint32_t)b->mask_words * 4, 16);
-    m.agent_off = m.rel_off + a * (uint32_t)(d.max_boxes > 0 ? d.max_boxes : 1) * 32;
-    m.misc_off = m.agent_off + a * (uint32_t)(kAgentRecVecs + kDdaVecs) * 16;
-    m.ov_off = m.misc_off + 16;
-    m.bytes = m.ov_off + a * (uint32_t)(d.max_overlay_rects > 0 ? d.max_overlay_rects : 1) * 32 +
-              round_up(a * ((ntiles + 31) / 32) * 4, 16);
+    m.agent_off = m.tile_off + ntiles * 16;
+    m.agent_ov_off = kAgentRelOff + (uint32_t)(d.max_boxes > 0 ? d.max_boxes : 1) * 32;
+    m.agent_mask_off = m.agent_ov_off + (uint32_t)(d.max_overlay_rects > 0 ? d.max_overlay_rects : 1) * 32;
+    m.agent_ovtile_off = m.agent_mask_off + round_up(ntiles * (uint32_t)b->mask_words * 4, 16);
+    m.agent_stride = m.agent_ovtile_off + round_up(((ntiles + 31) / 32) * 4, 16);
+    m.misc_off = m.agent_off + (uint32_t)apc * m.agent_stride;
+    m.bytes = m.misc_off + 16;
     return m;
+}
+
+// The three instantiations of the render kernel: column-word walk (grid at most 32 high, occupancy
+// staged), indexed walk with staged occupancy, indexed walk with the occupancy in global memory.
+using RenderFn = void (*)(const RenderParams);
+RenderFn render_fn(const mv_batch *b) {
+    if (!b->occ_shared) return render_kernel<kRenderThreads, false, false>;
+    return b->lay.ysh == 5 ? render_kernel<kRenderThreads, true, true> : render_kernel<kRenderThreads, true, false>;
 }
 
 int launch_render(mv_batch *b, uint8_t *d_rgb, float *d_depth, int obs_begin, int obs_count, cudaStream_t s) {
@@ -135,9 +144,10 @@ int launch_render(mv_batch *b, uint8_t *d_rgb, float *d_depth, int obs_begin, in
     p.sky_rgbx = b->sky_rgbx;
     p.miss_depth = b->desc.miss_depth;
     const uint32_t unstaged = b->occ_shared ? 0u : b->lay.occ_bytes;   // shared-memory offsets shift down by it
-    p.smem_tile_off = b->smem.tile_off - unstaged; p.smem_mask_off = b->smem.mask_off - unstaged;
-    p.smem_rel_off = b->smem.rel_off - unstaged; p.smem_agent_off = b->smem.agent_off - unstaged;
-    p.smem_misc_off = b->smem.misc_off - unstaged; p.smem_ov_off = b->smem.ov_off - unstaged;
+    p.smem_tile_off = b->smem.tile_off - unstaged; p.smem_agent_off = b->smem.agent_off - unstaged;
+    p.smem_misc_off = b->smem.misc_off - unstaged;
+    p.agent_stride = b->smem.agent_stride; p.agent_ov_off = b->smem.agent_ov_off;
+    p.agent_mask_off = b->smem.agent_mask_off; p.agent_ovtile_off = b->smem.agent_ovtile_off;
     p.agents_per_cta = b->agents_per_cta;
     p.max_steps = b->desc.grid_x + b->desc.grid_y + b->desc.grid_z + 3;
     // accumulated crossing times drift from the exact products by at most one rounding per step
@@ -148,10 +158,7 @@ int launch_render(mv_batch *b, uint8_t *d_rgb, float *d_depth, int obs_begin, in
     p.wait_polls = b->wait_polls;
     p.skip_staging = b->skip_staging;
     const int ctas = obs_count / b->agents_per_cta;   // callers pass whole environments when a CTA renders one
-    if (b->occ_shared)
-        render_kernel<kRenderThreads, true><<<ctas, kRenderThreads, b->smem.bytes, s>>>(p);
-    else
-        render_kernel<kRenderThreads, false><<<ctas, kRenderThreads, b->smem.bytes - b->lay.occ_bytes, s>>>(p);
+    render_fn(b)<<<ctas, kRenderThreads, b->smem.bytes - unstaged, s>>>(p);
     b->launches++;
     MV_CUDA(b, cudaGetLastError());
     return MV_OK;
@@ -331,10 +338,9 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
     if ((int)(b->smem.bytes - L.occ_bytes) > smem_max) { delete b; return MV_ERR_UNSUPPORTED; }
     // The dynamic shared-memory cap is a property of the kernel function on this device, shared by
     // every batch: raise it to the device's maximum once, never to one batch's own size.
-    e = cudaFuncSetAttribute(render_kernel<kRenderThreads, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(render_kernel<kRenderThreads, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 smem_max);
+    for (RenderFn f : {RenderFn(render_kernel<kRenderThreads, true, true>), RenderFn(render_kernel<kRenderThreads, true, false>),
+                       RenderFn(render_kernel<kRenderThreads, false, false>)})
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max);
     if (e != cudaSuccess) { delete b; return MV_ERR_CUDA; }
     // One CTA per environment (block staged once for all its agents) when that still fills the GPU;
     // otherwise one CTA per observation.  Cost model: waves of resident CTAs x (agents + fixed part).
@@ -344,11 +350,8 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
         if ((int)(all.bytes - unstaged) <= smem_max) {
             auto waves_cost = [&](const mv_batch::Smem &m, int apc) {
                 int per_sm = 0;
-                cudaError_t q = b->occ_shared
-                    ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, render_kernel<kRenderThreads, true>,
-                                                                    kRenderThreads, m.bytes)
-                    : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, render_kernel<kRenderThreads, false>,
-                                                                    kRenderThreads, m.bytes - L.occ_bytes);
+                cudaError_t q = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, render_fn(b), kRenderThreads,
+                                                                              m.bytes - unstaged);
                 if (q != cudaSuccess || per_sm < 1) return 1e30;
                 const double slots = (double)per_sm * sms, ctas = (double)b->num_obs / apc;
                 return std::ceil(ctas / slots) * (apc + kCtaFixedCost);

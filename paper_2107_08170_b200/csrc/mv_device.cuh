@@ -62,10 +62,11 @@ struct RenderParams {
     int agents_per_cta;                // observations one CTA renders: 1, or all agents of its env
     int max_steps;                     // bound of the traversal loop: grid_x + grid_y + grid_z + 3
     float exit_scale;                  // 1 - (bound on the rounding drift of accumulated crossing times)
-    // shared-memory offsets after the staged env block: tile table, per-agent box masks, per-agent
-    // eye-relative boxes, per-agent camera records + DDA start tables, barrier and flag words,
-    // per-agent overlay rectangles + touched-tile bits
-    uint32_t smem_tile_off, smem_mask_off, smem_rel_off, smem_agent_off, smem_misc_off, smem_ov_off;
+    // shared-memory offsets after the staged env block: tile table, per-agent blocks (camera record,
+    // DDA start table, eye-relative boxes, then overlay rectangles, per-tile box masks and per-tile
+    // overlay bits at the offsets below), barrier and flag words
+    uint32_t smem_tile_off, smem_agent_off, smem_misc_off;
+    uint32_t agent_stride, agent_ov_off, agent_mask_off, agent_ovtile_off;
     const int4 *overlay;               // [O][max_overlay] 16-byte records, or null
     const int32_t *overlay_count;      // [O]
     int max_overlay;

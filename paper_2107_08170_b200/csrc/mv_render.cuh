@@ -74,81 +74,85 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
     return r;
 }
 
-// The DDA loop (see render_kernel).  Operands: %0 voxel index (in/out), %1 hit time (in/out: kept
-// unless a filled cell is entered), %2 = shared-memory address of the colour-table row of the face
-// entered at a hit (in/out, kept likewise), %3..%5 = crossing times per axis (in/out), %6..%8 = dt per
-// axis, %9..%11 = index strides, %12 = exit time, %13 = step budget, %14 = shared-memory
-// address of the ray's DDA table rows (whose fourth words are the colour-table rows per axis),
-// %15 = 64-bit global base of the occupancy words (only when they are not staged in shared memory).
-// One step: t = min(tx,ty,tz); leave when t >= exit time or when the cell entered by the previous step
-// is filled (one branch for both); else the axis whose crossing time equals t (ties: x, then y, then
-// z) advances: crossing time += dt, voxel index += stride; then the new cell's occupancy bit is
-// tested.  Two registers alternate as t, so that after a hit the time at which the filled cell was
-// entered is still there.  The voxel index carries 8x the shared-memory byte address of the occupancy
-// grid, so (index >> 3) & ~3 is the word's address and index & 31 the bit (the index is
-// ((x + grid_x*z) << ysh) | y: steps along x and z change the word, steps along y the bit).
+// ---------------------------------------------------------------------------------------------
+// The DDA loop.  Crossing times accumulate (t += dt) and the exit time handed in is pulled in by
+// the rounding drift that can build up, which keeps the walk inside the occupied box; the loop is
+// also bounded by a step budget.  One step: t = min(tx,ty,tz); leave when t >= exit time or when
+// the cell entered by the previous step is filled (one branch for both); else the axis whose
+// crossing time equals t (ties: x, then y, then z) advances.  Two registers alternate as t, so
+// that after a hit the time at which the filled cell was entered is still there.
+//
+// Two flavours of the cell state:
+//  * column-word (grids up to 32 voxels high, occupancy in shared memory): the state is the
+//    shared-memory address `pos` of the (x, z) column's word and a one-bit mask `bit` of the height;
+//    x and z steps add a byte stride to the address, a y step rotates the mask by 1 or 31, and the
+//    test is one load and one AND.
+//  * indexed (any grid): the state is the voxel index `pos` (plus 8x the shared-memory byte address
+//    of the occupancy when it is staged, so that (pos >> 3) & ~3 is the word's address and pos & 31
+//    the bit); every step adds a stride.
+// Register names used by the macros (declared by the enclosing asm block): tx ty tz dtx dty dtz
+// (f32), sx sy sz pos bit w a it (b32), ta tb (f32), px py pz pq ph pf (pred), texit (f32); the
+// global flavour also uses ag (b64) and the operand named by MV_DDA_GBASE.
 #if defined(MV_PROBE) && MV_PROBE == 9
 #define MV_DDA_COUNT " add.f32 ns, ns, 0f3F800000;\n"
-#define MV_DDA_COUNT_OUT " mov.f32 %1, ns;\n"
 #else
 #define MV_DDA_COUNT
-#define MV_DDA_COUNT_OUT
 #endif
-#define MV_DDA_ADVANCE(T, OUT)                       \
-    " min.f32 " T ", %3, %4, %5;\n"                  \
-    " setp.geu.or.f32 pq, " T ", %12, ph;\n"         \
+#if defined(MV_TEST_FORM) && MV_TEST_FORM == 1
+#define MV_DDA_TESTBIT " and.b32 w, w, bit;\n setp.ne.u32 ph, w, 0;\n"
+#else
+#define MV_DDA_TESTBIT " lop3.or.b32 w|ph, w, bit, 0, 0xC0, pf;\n"
+#endif
+#define MV_DDA_HEAD(T, OUT)                          \
+    " min.f32 " T ", tx, ty, tz;\n"                  \
+    " setp.geu.or.f32 pq, " T ", texit, ph;\n"       \
     " @pq bra " OUT ";\n"                            \
     MV_DDA_COUNT                                     \
-    " setp.eq.f32 px, %3, " T ";\n"                  \
-    " setp.eq.and.f32 py|pz, %4, " T ", !px;\n"      \
-    " @px add.f32 %3, %3, %6;\n"                     \
-    " @px add.s32 %0, %0, %9;\n"                     \
-    " @py add.f32 %4, %4, %7;\n"                     \
-    " @py add.s32 %0, %0, %10;\n"                    \
-    " @pz add.f32 %5, %5, %8;\n"                     \
-    " @pz add.s32 %0, %0, %11;\n"
-#define MV_DDA_TEST                                  \
-    " shf.r.wrap.b32 w, w, 0, %0;\n"                 \
-    " and.b32 w, w, 1;\n"                            \
-    " setp.ne.u32 ph, w, 0;\n"
-#define MV_DDA_LOAD_SHARED " shr.u32 a, %0, 3;\n and.b32 a, a, 0xfffffffc;\n ld.shared.u32 w, [a];\n"
-#define MV_DDA_LOAD_GLOBAL " shr.u32 a, %0, 5;\n mad.wide.u32 ag, a, 4, %15;\n ld.global.nc.u32 w, [ag];\n"
-#define MV_DDA_STEP(T, OUT) MV_DDA_ADVANCE(T, OUT) MV_DDA_LOAD_SHARED MV_DDA_TEST
-#define MV_DDA_STEP_GLOBAL(T, OUT) MV_DDA_ADVANCE(T, OUT) MV_DDA_LOAD_GLOBAL MV_DDA_TEST
-#define MV_DDA_PROLOGUE                              \
-    "{\n"                                            \
-    " .reg .pred px, py, pz, pq, ph;\n"              \
-    " .reg .f32 ta, tb, ns;\n"                       \
-    " .reg .u32 w, a;\n"                             \
-    " .reg .u64 ag;\n"                               \
-    " .reg .s32 it;\n"                               \
-    " mov.s32 it, %13;\n"                            \
-    " mov.f32 ns, 0f00000000;\n"                     \
-    " mov.f32 tb, 0f00000000;\n"                     \
+    " setp.eq.f32 px, tx, " T ";\n"                  \
+    " setp.eq.and.f32 py|pz, ty, " T ", !px;\n"      \
+    " @px add.f32 tx, tx, dtx;\n"                    \
+    " @py add.f32 ty, ty, dty;\n"                    \
+    " @pz add.f32 tz, tz, dtz;\n"
+#define MV_DDA_STEP_COLW(T, OUT) MV_DDA_HEAD(T, OUT)  \
+    " @px add.s32 pos, pos, sx;\n"                   \
+    " @pz add.s32 pos, pos, sz;\n"                   \
+    " @py shf.l.wrap.b32 bit, bit, bit, sy;\n"       \
+    " ld.shared.u32 w, [pos];\n"                     \
+    MV_DDA_TESTBIT
+#define MV_DDA_STEP_IDX_TAIL                         \
+    " shf.r.wrap.b32 w, w, 0, pos;\n"                \
+    " lop3.or.b32 w|ph, w, 1, 0, 0xC0, pf;\n"
+#define MV_DDA_STEP_IDX_ADV                          \
+    " @px add.s32 pos, pos, sx;\n"                   \
+    " @py add.s32 pos, pos, sy;\n"                   \
+    " @pz add.s32 pos, pos, sz;\n"
+#define MV_DDA_STEP_IDX(T, OUT) MV_DDA_HEAD(T, OUT) MV_DDA_STEP_IDX_ADV \
+    " shr.u32 a, pos, 3;\n and.b32 a, a, 0xfffffffc;\n ld.shared.u32 w, [a];\n" MV_DDA_STEP_IDX_TAIL
+#define MV_DDA_STEP_IDX_GLOBAL(T, OUT) MV_DDA_HEAD(T, OUT) MV_DDA_STEP_IDX_ADV \
+    " shr.u32 a, pos, 5;\n mad.wide.u32 ag, a, 4, gbase;\n ld.global.nc.u32 w, [ag];\n" MV_DDA_STEP_IDX_TAIL
+// Loop around four steps.  On leaving: ph = a filled cell was entered, thit = when, and px/py
+// still say along which axis.
+#define MV_DDA_LOOP(STEP)                            \
+    " setp.ne.u32 pf, 0, 0;\n"                       \
     " setp.ne.u32 ph, 0, 0;\n"                       \
-    " setp.ne.u32 px, 0, 0;\n"                       \
-    " setp.ne.u32 py, 0, 0;\n"                       \
-    "MV_DDA_LOOP:\n"
-#define MV_DDA_EPILOGUE                              \
+    " mov.f32 tb, 0f00000000;\n"                     \
+    "MV_DDA_LOOP_TOP:\n"                             \
+    STEP("ta", "MV_DDA_OUT_A") STEP("tb", "MV_DDA_OUT_B") STEP("ta", "MV_DDA_OUT_A") STEP("tb", "MV_DDA_OUT_B") \
     " sub.s32 it, it, 4;\n"                          \
-    " setp.gt.s32 pq, it, 0;\n"                     \
-    " @pq bra MV_DDA_LOOP;\n"                        \
+    " setp.gt.s32 pq, it, 0;\n"                      \
+    " @pq bra MV_DDA_LOOP_TOP;\n"                    \
     "MV_DDA_OUT_A:\n"                                \
-    " @ph mov.f32 %1, tb;\n"                         \
+    " @ph mov.f32 thit, tb;\n"                       \
     " bra MV_DDA_OUT;\n"                             \
     "MV_DDA_OUT_B:\n"                                \
-    " @ph mov.f32 %1, ta;\n"                         \
-    "MV_DDA_OUT:\n"                                  \
-    " selp.u32 a, 16, 32, py;\n"                     \
-    " selp.u32 a, 0, a, px;\n"                       \
-    " add.u32 a, a, %14;\n"                          \
-    " @ph ld.shared.u32 %2, [a+12];\n"               \
-    MV_DDA_COUNT_OUT                                 \
-    "}\n"
-#define MV_DDA_BODY MV_DDA_PROLOGUE MV_DDA_STEP("ta", "MV_DDA_OUT_A") MV_DDA_STEP("tb", "MV_DDA_OUT_B") \
-    MV_DDA_STEP("ta", "MV_DDA_OUT_A") MV_DDA_STEP("tb", "MV_DDA_OUT_B") MV_DDA_EPILOGUE
-#define MV_DDA_BODY_GLOBAL MV_DDA_PROLOGUE MV_DDA_STEP_GLOBAL("ta", "MV_DDA_OUT_A") MV_DDA_STEP_GLOBAL("tb", "MV_DDA_OUT_B") \
-    MV_DDA_STEP_GLOBAL("ta", "MV_DDA_OUT_A") MV_DDA_STEP_GLOBAL("tb", "MV_DDA_OUT_B") MV_DDA_EPILOGUE
+    " @ph mov.f32 thit, ta;\n"                       \
+    "MV_DDA_OUT:\n"
+#define MV_DDA_DECL                                  \
+    " .reg .pred px, py, pz, pq, ph, pf;\n"          \
+    " .reg .f32 tx, ty, tz, dtx, dty, dtz, ta, tb, texit, thit, ns;\n" \
+    " .reg .b32 sx, sy, sz, pos, bit, w, a, it;\n"   \
+    " .reg .b64 ag, gbase;\n"                        \
+    " mov.f32 ns, 0f00000000;\n"
 
 #ifndef MV_PROBE
 #define MV_PROBE 0
@@ -159,15 +163,41 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
 
 constexpr uint32_t kAgentInside = 1u;      // eye inside the occupied cell box
 constexpr uint32_t kAgentBad = 2u;         // non-finite camera: sky frame
-constexpr int kAgentRecVecs = 4;           // float4 slots per agent: camera (3) + {start index, flags, self box, overlay count}
-constexpr int kDdaVecs = 24;               // float4 slots per agent: 8 sign combinations x 3 axes
+constexpr uint32_t kAgentFilled = 4u;      // the eye's own voxel is filled
+// Per-agent block in shared memory (16-byte slots): camera record (3), {-, flags, self box, overlay
+// count} (1), {start bit mask, exit-time factor, start colour row, start position} (1), {64-bit address
+// of the env's material store, biased for the walk's positions} (1), DDA start
+// table (8 sign combinations x 3 axes), then eye-relative boxes, overlay rectangles, per-tile box
+// masks and per-tile overlay bits at offsets the host lays out.
+constexpr int kAgentRecVecs = 6;
+constexpr int kDdaVecs = 24;
+// byte offsets, from the agent block's start plus 48 x (sign combination), of the DDA table rows of
+// the x, y and z axis and of the colour-row word of the x row (as text, for the PTX blocks)
+// hard bound of the traversal loop: no grid allows more steps than 3 x 1024 + 3
+#define MV_STEP_BUDGET "3080"
+#define MV_TAB_X "96"
+#define MV_TAB_Y "112"
+#define MV_TAB_Z "128"
+#define MV_TAB_ROW "108"
+static_assert(16 * kAgentRecVecs == 96, "MV_TAB_* follow the agent record size");
+constexpr uint32_t kAgentDdaOff = 16u * kAgentRecVecs;
+constexpr uint32_t kAgentRelOff = 16u * (kAgentRecVecs + kDdaVecs);
+
+// One thread's share of a sky frame (non-finite camera).
+template <int NT>
+__device__ __forceinline__ void write_sky(uint8_t *rgb_obs, float *depth_obs, int npx, uint32_t sky_rgbx, float miss_depth) {
+    for (int i = threadIdx.x; i < npx; i += NT) depth_obs[i] = miss_depth;
+    for (int i = threadIdx.x; i < npx * 3; i += NT) rgb_obs[i] = (uint8_t)(sky_rgbx >> (8 * (i % 3)));
+}
 
 // OCC_SHARED: the occupancy bits are staged in shared memory with the rest of the env block (the
 // normal case); otherwise only the block's tail (colour table, boxes, bounds) is staged and the
 // occupancy is read from global memory through the read-only path.
-template <int NT, bool OCC_SHARED>
+// COLW: column-word flavour of the walk (grid at most 32 high and occupancy staged).
+template <int NT, bool OCC_SHARED, bool COLW>
 __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams p)
 {
+    static_assert(OCC_SHARED || !COLW, "the column-word walk reads shared memory");
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int apc = p.agents_per_cta;
@@ -186,16 +216,16 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     const float4 *s_box = reinterpret_cast<const float4 *>(smem + (p.lay.box_off - unstaged));
     const int *s_count = reinterpret_cast<const int *>(smem + (p.lay.count_off - unstaged));
     float4 *s_tile = reinterpret_cast<float4 *>(smem + p.smem_tile_off);
-    uint32_t *s_mask = reinterpret_cast<uint32_t *>(smem + p.smem_mask_off);
-    float4 *s_rel = reinterpret_cast<float4 *>(smem + p.smem_rel_off);
-    float4 *s_agent = reinterpret_cast<float4 *>(smem + p.smem_agent_off);
-    float4 *s_dda = s_agent + apc * kAgentRecVecs;
+    unsigned char *s_agents = smem + p.smem_agent_off;
     uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem + p.smem_misc_off);
     uint32_t *s_flag = reinterpret_cast<uint32_t *>(smem + p.smem_misc_off + 8);
-    int4 *s_ov = reinterpret_cast<int4 *>(smem + p.smem_ov_off);
-    const int ov_slots = 2 * max(p.max_overlay, 1);                 // int4 slots per agent
+    auto agent_rec = [&](int ag) { return reinterpret_cast<float4 *>(s_agents + (size_t)ag * p.agent_stride); };
+    auto agent_dda = [&](int ag) { return agent_rec(ag) + kAgentRecVecs; };
+    auto agent_rel = [&](int ag) { return agent_rec(ag) + kAgentRecVecs + kDdaVecs; };
+    auto agent_ov = [&](int ag) { return reinterpret_cast<int4 *>(s_agents + (size_t)ag * p.agent_stride + p.agent_ov_off); };
+    auto agent_mask = [&](int ag) { return reinterpret_cast<uint32_t *>(s_agents + (size_t)ag * p.agent_stride + p.agent_mask_off); };
+    auto agent_ovtile = [&](int ag) { return reinterpret_cast<uint32_t *>(s_agents + (size_t)ag * p.agent_stride + p.agent_ovtile_off); };
     const int ovt_words = (ntiles + 31) / 32;
-    uint32_t *s_ovtile = reinterpret_cast<uint32_t *>(s_ov + apc * ov_slots);
 
     // ---- stage the environment block
     if (tid == 0) mbar_init(s_bar, 1);
@@ -205,7 +235,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         bulk_load(smem, env_block + unstaged, p.lay.block_bytes - unstaged, s_bar);
     }
     // ---- meanwhile: tile table, cleared masks, camera records, GUI rectangles
-    for (int i = tid; i < apc * ntiles * mw; i += NT) s_mask[i] = 0u;
+    for (int i = tid; i < apc * ntiles * mw; i += NT) agent_mask(i / (ntiles * mw))[i % (ntiles * mw)] = 0u;
     for (int i = tid; i < ntiles; i += NT) {
         const int ty = i / p.tiles_x, tx = i - ty * p.tiles_x;
         // a = 2px+1-W and b = H-1-2py of the tile's first pixel (small integers: exact as floats)
@@ -215,18 +245,18 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     if (tid < apc) {
         const float4 *cq = reinterpret_cast<const float4 *>(p.cams + obs0 + tid);
         const float4 c3 = __ldg(cq + 3);
-        s_agent[kAgentRecVecs * tid + 0] = __ldg(cq);
-        s_agent[kAgentRecVecs * tid + 1] = __ldg(cq + 1);
-        s_agent[kAgentRecVecs * tid + 2] = __ldg(cq + 2);
+        float4 *rec = agent_rec(tid);
+        rec[0] = __ldg(cq);
+        rec[1] = __ldg(cq + 1);
+        rec[2] = __ldg(cq + 2);
         const int ovc = p.overlay ? min(max(__ldg(p.overlay_count + obs0 + tid), 0), p.max_overlay) : 0;
-        // slot 3: {start voxel index (filled in below), flags, self box, overlay count}
-        s_agent[kAgentRecVecs * tid + 3] = make_float4(0.0f, __uint_as_float((__float_as_uint(c3.y) & kFlagBadCamera) ? kAgentBad : 0u),
-                                                        c3.x, __int_as_float(ovc));
+        rec[3] = make_float4(0.0f, __uint_as_float((__float_as_uint(c3.y) & kFlagBadCamera) ? kAgentBad : 0u), c3.x,
+                             __int_as_float(ovc));
     }
     if (p.overlay) {
         // GUI rectangles of each observation (unpacked to x0,y0,x1,y1 / colour in two slots) and one
         // bit per tile that any rectangle touches, so untouched tiles pay a single bit test
-        for (int i = tid; i < apc * ovt_words; i += NT) s_ovtile[i] = 0u;
+        for (int i = tid; i < apc * ovt_words; i += NT) agent_ovtile(i / ovt_words)[i % ovt_words] = 0u;
         __syncthreads();
         for (int i = tid; i < apc * p.max_overlay; i += NT) {
             const int ag = i / p.max_overlay, r = i - ag * p.max_overlay;
@@ -235,14 +265,14 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             const int4 q = __ldg(p.overlay + (size_t)(obs0 + ag) * p.max_overlay + r);
             const int x0 = (int)(short)(q.x & 0xffff), y0 = (int)(short)(q.x >> 16);
             const int x1 = (int)(short)(q.y & 0xffff), y1 = (int)(short)(q.y >> 16);
-            s_ov[ag * ov_slots + 2 * r] = make_int4(x0, y0, x1, y1);
-            s_ov[ag * ov_slots + 2 * r + 1] = make_int4(q.z & 0xffffff, 0, 0, 0);
+            agent_ov(ag)[2 * r] = make_int4(x0, y0, x1, y1);
+            agent_ov(ag)[2 * r + 1] = make_int4(q.z & 0xffffff, 0, 0, 0);
             const int cx0 = max(x0, 0), cy0 = max(y0, 0), cx1 = min(x1, W), cy1 = min(y1, H);
             if (cx0 < cx1 && cy0 < cy1)
                 for (int ty = cy0 >> 2; ty <= ((cy1 - 1) >> 2); ++ty)
                     for (int tx = cx0 >> 3; tx <= ((cx1 - 1) >> 3); ++tx) {
                         const int t = ty * p.tiles_x + tx;
-                        atomicOr(&s_ovtile[ag * ovt_words + (t >> 5)], 1u << (t & 31));
+                        atomicOr(&agent_ovtile(ag)[t >> 5], 1u << (t & 31));
                     }
         }
     }
@@ -265,23 +295,35 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     // ---- per-agent traversal set-up and box binning
     const int gx = p.gx, gz = p.gz;
     // voxel-index strides of the y-packed layout: x and z move by whole columns, y by single bits
-    const int stride_x = 1 << p.lay.ysh, stride_z = gx << p.lay.ysh, stride_y = 1;
+    const int stride_x = 1 << p.lay.ysh, stride_z = gx << p.lay.ysh;
     // Traversal is confined to the cell box [lo, hi) that holds every filled voxel of this env
     // (nothing outside it can be hit), so rays that leave it, e.g. into the sky, stop there.
     const int lox = s_count[1], loy = s_count[2], loz = s_count[3];
     const int hix = s_count[4], hiy = s_count[5], hiz = s_count[6];
     const bool any_voxel = (lox < hix) && (loy < hiy) && (loz < hiz);
-    const uint32_t vi_bias = OCC_SHARED ? 8u * smem_addr(smem) : 0u;
+    const uint32_t occ_base = OCC_SHARED ? smem_addr(smem) : 0u;
+    const uint32_t vi_bias = 8u * occ_base;
     const int P_ = p.palette;
     const uint32_t lut_base = smem_addr(s_lut);
+    const uint32_t inside_row = lut_base + (uint32_t)(kFaceInside * P_ * 4);
+    // position of cell (cx, cy, cz) in the walk's own terms (see MV_DDA_*)
+    auto cell_pos = [&](int cx, int cy, int cz) -> uint32_t {
+        return COLW ? occ_base + 4u * (uint32_t)(cx + gx * cz) : vi_bias + (uint32_t)(stride_x * cx + stride_z * cz + cy);
+    };
+    auto cell_filled = [&](int cx, int cy, int cz) -> bool {
+        const uint32_t u = (uint32_t)(stride_x * cx + stride_z * cz + cy);
+        return (s_occ[u >> 5] >> (u & 31)) & 1u;
+    };
     if (tid < kDdaVecs * apc) {
         // DDA start table of agent ag, entry 3*signs + axis (bit c of `signs` set: direction component c
         // negative): x = signed distance from the eye to the cell face the ray meets first, y = cells
-        // left before the occupied box ends that way, z = voxel-index stride, w = shared-memory address
-        // of the colour-table row of the face entered by a step along this axis.
+        // left before the occupied box ends that way, z = what a step along the axis adds to the
+        // position (column-word flavour: byte stride for x and z, rotate count for y), w = shared-memory
+        // address of the colour-table row of the face entered by a step along this axis.
         const int ag = tid / kDdaVecs, e = tid - ag * kDdaVecs;
         const int signs = e / 3, ax = e - 3 * signs, neg = (signs >> ax) & 1;
-        const float4 c0 = s_agent[kAgentRecVecs * ag];
+        float4 *rec = agent_rec(ag);
+        const float4 c0 = rec[0];
         const float Pc = ax == 0 ? c0.x : (ax == 1 ? c0.y : c0.z);
         const bool cam_in = any_voxel && (c0.x >= (float)lox) && (c0.x < (float)hix) && (c0.y >= (float)loy) &&
                             (c0.y < (float)hiy) && (c0.z >= (float)loz) && (c0.z < (float)hiz);
@@ -289,28 +331,35 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         if (cam_in) { cx0 = (int)floorf(c0.x); cy0 = (int)floorf(c0.y); cz0 = (int)floorf(c0.z); }
         const int cc = ax == 0 ? cx0 : (ax == 1 ? cy0 : cz0);
         const int lo_c = ax == 0 ? lox : (ax == 1 ? loy : loz), hi_c = ax == 0 ? hix : (ax == 1 ? hiy : hiz);
-        const int st = ax == 0 ? stride_x : (ax == 1 ? stride_y : stride_z);
-        s_dda[kDdaVecs * ag + e] = make_float4(neg ? (float)cc - Pc : (float)(cc + 1) - Pc,
-                                               neg ? (float)(cc - lo_c) : (float)(hi_c - 1 - cc),
-                                               __int_as_float(neg ? -st : st),
-                                               __uint_as_float(lut_base + (uint32_t)((2 * ax + neg) * P_ * 4)));
+        int st;
+        if (COLW) st = ax == 0 ? (neg ? -4 : 4) : (ax == 1 ? (neg ? 31 : 1) : (neg ? -4 * gx : 4 * gx));
+        else st = (ax == 0 ? stride_x : (ax == 1 ? 1 : stride_z)) * (neg ? -1 : 1);
+        agent_dda(ag)[e] = make_float4(neg ? (float)cc - Pc : (float)(cc + 1) - Pc,
+                                       neg ? (float)(cc - lo_c) : (float)(hi_c - 1 - cc), __int_as_float(st),
+                                       __uint_as_float(lut_base + (uint32_t)((2 * ax + neg) * P_ * 4)));
         if (e == 0) {
-            const int vi0 = stride_x * cx0 + stride_z * cz0 + stride_y * cy0;
-            const bool filled = cam_in && ((s_occ[vi0 >> 5] >> (vi0 & 31)) & 1u);
-            float4 *slot = &s_agent[kAgentRecVecs * ag + 3];
-            slot->x = __uint_as_float((uint32_t)vi0 + vi_bias);
-            slot->y = __uint_as_float(__float_as_uint(slot->y) | (cam_in ? kAgentInside : 0u) | (filled ? 4u : 0u));
+            const bool filled = cam_in && cell_filled(cx0, cy0, cz0);
+            rec[3].y = __uint_as_float(__float_as_uint(rec[3].y) | (cam_in ? kAgentInside : 0u) | (filled ? kAgentFilled : 0u));
+            // exit-time factor: pulls the exit in by the rounding drift of the accumulated crossing
+            // times; -inf (the product is then -inf or NaN and the first test ends the walk) when the
+            // eye sits in a filled voxel
+            rec[4] = make_float4(__uint_as_float(1u << cy0), filled ? -kInf : p.exit_scale,
+                                 __uint_as_float(filled ? inside_row : kNoRow), __uint_as_float(cell_pos(cx0, cy0, cz0)));
+            const unsigned long long mp = reinterpret_cast<unsigned long long>(
+                p.mat + (size_t)env * ((size_t)gx * gz << p.lay.ysh) - vi_bias);
+            rec[5] = make_float4(__uint_as_float((uint32_t)mp), __uint_as_float((uint32_t)(mp >> 32)),
+                                 __uint_as_float(p.sky_rgbx), p.miss_depth);
         }
     }
     {
         const int nb = min(s_count[0], p.max_boxes);
         for (int i = tid; i < apc * p.max_boxes; i += NT) {
             const int ag = i / p.max_boxes, b = i - ag * p.max_boxes;
-            const float4 c0 = s_agent[kAgentRecVecs * ag], c1 = s_agent[kAgentRecVecs * ag + 1];
-            const float4 c2 = s_agent[kAgentRecVecs * ag + 2];
+            const float4 *rec = agent_rec(ag);
+            const float4 c0 = rec[0], c1 = rec[1], c2 = rec[2];
             const float Px = c0.x, Py = c0.y, Pz = c0.z, Fx = c0.w, Fy = c1.x, Fz = c1.y;
             const float Rx = c1.z, Ry = c1.w, Rz = c2.x, Ux = c2.y, Uy = c2.z, Uz = c2.w;
-            const int self_box = __float_as_int(s_agent[kAgentRecVecs * ag + 3].z);
+            const int self_box = __float_as_int(rec[3].z);
             const float r2 = Rx * Rx + Ry * Ry + Rz * Rz, u2 = Ux * Ux + Uy * Uy + Uz * Uz;
             const float ir2 = 1.0f / r2, iu2 = 1.0f / u2;
             const float4 A = s_box[2 * b], B = s_box[2 * b + 1];
@@ -332,8 +381,8 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                 fymin = fminf(fymin, fy); fymax = fmaxf(fymax, fy);
             }
             const bool front = tmin > 0.05f;                 // whole box safely in front of the eye plane
-            s_rel[2 * i] = make_float4(lx, ly, lz, front ? tmin * 0.9999f : 0.0f);
-            s_rel[2 * i + 1] = make_float4(hx, hy, hz, B.z);
+            agent_rel(ag)[2 * b] = make_float4(lx, ly, lz, front ? tmin * 0.9999f : 0.0f);
+            agent_rel(ag)[2 * b + 1] = make_float4(hx, hy, hz, B.z);
             if (!valid || tmax < -1e-3f) continue;           // ignored, or wholly behind the eye
             int px0 = 0, px1 = W - 1, py0 = 0, py1 = H - 1;
             if (front) {
@@ -344,7 +393,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                 if (px0 > px1 || py0 > py1) continue;
             }
             const uint32_t bit = 1u << (b & 31);
-            uint32_t *mask = s_mask + (size_t)ag * ntiles * mw;
+            uint32_t *mask = agent_mask(ag);
             for (int ty = py0 >> 2; ty <= (py1 >> 2); ++ty)
                 for (int tx = px0 >> 3; tx <= (px1 >> 3); ++tx)
                     atomicOr(&mask[(ty * p.tiles_x + tx) * mw + (b >> 5)], bit);
@@ -352,7 +401,6 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     }
     __syncthreads();
 
-    const uint8_t *mat_env = p.mat + (size_t)env * ((size_t)gx * gz << p.lay.ysh) - vi_bias;
     const float flox = (float)lox, floy = (float)loy, floz = (float)loz;
     const float fhix = (float)hix, fhiy = (float)hiy, fhiz = (float)hiz;
 
@@ -373,186 +421,279 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     const int rgb_lane_off = st_r * W * 3 + st_j * 4;
     keep(lane_a); keep(lane_b); keep(st_src); keep(st_sel);
     const uint32_t tile_begin = smem_addr(s_tile) + 16u * (uint32_t)warp;
+#if MV_PROBE == 3
+    const uint32_t tile_end = smem_addr(s_tile);
+#else
     const uint32_t tile_end = smem_addr(s_tile) + 16u * (uint32_t)ntiles;
-    const uint32_t inside_row = lut_base + (uint32_t)(kFaceInside * P_ * 4);
+#endif
 
     for (int ag = 0; ag < apc; ++ag) {
         const int obs = obs0 + ag;
         uint8_t *rgb_obs = p.rgb + (size_t)obs * H * W * 3;
         float *depth_obs = p.depth + (size_t)obs * H * W;
-        const float4 c0 = s_agent[kAgentRecVecs * ag], c1 = s_agent[kAgentRecVecs * ag + 1];
-        const float4 c2 = s_agent[kAgentRecVecs * ag + 2], c3 = s_agent[kAgentRecVecs * ag + 3];
+        const float4 c0 = agent_rec(ag)[0], c3 = agent_rec(ag)[3];
         const uint32_t aflags = __float_as_uint(c3.y);
         if (aflags & kAgentBad) {                   // non-finite camera: a sky frame
-            for (int i = tid; i < W * H; i += NT) depth_obs[i] = p.miss_depth;
-            for (int i = tid; i < W * H * 3; i += NT) rgb_obs[i] = (uint8_t)(p.sky_rgbx >> (8 * (i % 3)));
+            write_sky<NT>(rgb_obs, depth_obs, W * H, p.sky_rgbx, p.miss_depth);
             continue;
         }
         const float Px = c0.x, Py = c0.y, Pz = c0.z;
         const bool cam_in = (aflags & kAgentInside) != 0;
-        uint32_t vi0 = __float_as_uint(c3.x);
-        const uint32_t row0 = (aflags & 4u) ? inside_row : kNoRow;
-        // exit-time factor: pulls the exit in by the rounding drift of the accumulated crossing times;
-        // -inf (so that the product is -inf or NaN and the first test ends the walk) when the eye sits
-        // in a filled voxel
-        float escale = (aflags & 4u) ? -kInf : p.exit_scale;
         const int ov_count = __float_as_int(c3.w);
-        uint32_t dda_base = smem_addr(s_dda + kDdaVecs * ag);
-        uint32_t mask_p = smem_addr(s_mask + ((size_t)ag * ntiles + warp) * mw);
-        const float4 *rel = s_rel + (size_t)ag * 2 * p.max_boxes;
-        const int4 *ov = s_ov + ag * ov_slots;
-        const uint32_t *ovtile = s_ovtile + ag * ovt_words;
-        float *depth_lane = depth_obs + depth_lane_off;
-        uint8_t *rgb_lane = rgb_obs + rgb_lane_off;
-        keep(vi0); keep(escale); keep64(depth_lane); keep64(rgb_lane);
-        const uint8_t *mat_lane = mat_env;
-        const uint32_t cam_p = smem_addr(s_agent + kAgentRecVecs * ag);
+        uint32_t abase = smem_addr(agent_rec(ag));
+        uint32_t mask_p = smem_addr(agent_mask(ag) + (size_t)warp * mw);
+        // (store addresses as global-space addresses for the PTX store block)
+        unsigned long long depth_lane = (unsigned long long)__cvta_generic_to_global(depth_obs + depth_lane_off);
+        unsigned long long rgb_lane = (unsigned long long)__cvta_generic_to_global(rgb_obs + rgb_lane_off);
+        keep(abase);
+        asm volatile("" : "+l"(depth_lane), "+l"(rgb_lane));
 
         // ---- tiles: warp w takes tiles w, w + nwarps, ... (8 x 4 pixels, one per lane)
         for (uint32_t tile_p = tile_begin; tile_p < tile_end; tile_p += 16u * kWarps, mask_p += 4u * kWarps * (uint32_t)mw) {
-            float Ta, Tb;
             int tile_px;
-            uint32_t tile_no;
-            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=f"(Ta), "=f"(Tb), "=r"(tile_px), "=r"(tile_no) : "r"(tile_p));
-            // ---- ray through the pixel centre: d = F + a*Rs + b*Us, a = 2px+1-W, b = H-1-2py
-            // (the basis is re-read from shared memory per tile: three broadcast loads cost less than
-            // nine registers held across the walk)
-            float Fx, Fy, Fz, Rx, Ry, Rz, Ux, Uy, Uz, unused;
-            asm volatile("ld.shared.f32 %0, [%1+12];" : "=f"(Fx) : "r"(cam_p));
-            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4+16];" : "=f"(Fy), "=f"(Fz), "=f"(Rx), "=f"(Ry) : "r"(cam_p));
-            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4+32];" : "=f"(Rz), "=f"(Ux), "=f"(Uy), "=f"(Uz) : "r"(cam_p));
-            (void)unused;
-            const float a = Ta + lane_a, bb = Tb - lane_b;
-            float dx = fmaf(bb, Ux, fmaf(a, Rx, Fx));
-            float dy = fmaf(bb, Uy, fmaf(a, Ry, Fy));
-            float dz = fmaf(bb, Uz, fmaf(a, Rz, Fz));
-            // a component that is exactly zero never crosses a cell face; 1e-30 keeps it that way
-            // without infinities in the slab arithmetic
-            dx = dx == 0.0f ? 1e-30f : dx;
-            dy = dy == 0.0f ? 1e-30f : dy;
-            dz = dz == 0.0f ? 1e-30f : dz;
-            const float ix = fast_rcp(dx), iy = fast_rcp(dy), iz = fast_rcp(dz);
-            const float dtx = fabsf(ix), dty = fabsf(iy), dtz = fabsf(iz);
-            const uint32_t sgn3 = (__float_as_uint(dx) >> 31) | ((__float_as_uint(dy) >> 30) & 2u) |
-                                  ((__float_as_uint(dz) >> 29) & 4u);      // bit c set: component c negative
-            const uint32_t tab = dda_base + 48u * sgn3;
-            // rows of the DDA table for this ray's signs: {distance to the first face, cells left, index
-            // stride, colour-table row} per axis; the colour-table rows are fetched only where needed
-            float qxx, qxy, qyx, qyy, qzx, qzy;
-            int sx, sy, sz;
-            {
-                uint32_t u0, u1, u2;
-                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=f"(qxx), "=f"(qxy), "=r"(sx), "=r"(u0) : "r"(tab));
-                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4+16];" : "=f"(qyx), "=f"(qyy), "=r"(sy), "=r"(u1) : "r"(tab));
-                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4+32];" : "=f"(qzx), "=f"(qzy), "=r"(sz), "=r"(u2) : "r"(tab));
-            }
-            auto face_row = [&](int axis) {            // colour-table row of the face entered along `axis`
-                uint32_t r;
-                asm volatile("ld.shared.u32 %0, [%1+12];" : "=r"(r) : "r"(tab + 16u * (uint32_t)axis));
-                return r;
-            };
-
-            // ---- start of the walk: cell, first crossing times, time at which the ray leaves the box
-            float t0x, t0y, t0z, t_exit, t_hit = 0.0f;
-            uint32_t vi = vi0, row = row0;
-            if (cam_in) {
-                t0x = qxx * ix;
-                t0y = qyx * iy;
-                t0z = qzx * iz;
-                t_exit = min3f(fmaf(qxy, dtx, t0x), fmaf(qyy, dty, t0y), fmaf(qzy, dtz, t0z)) * escale;
-            } else {
-                // eye outside the occupied box: clip the ray to it, start in the entry cell
-                const bool ngx = dx < 0.0f, ngy = dy < 0.0f, ngz = dz < 0.0f;
-                const float x1 = (flox - Px) * ix, x2 = (fhix - Px) * ix;
-                const float y1 = (floy - Py) * iy, y2 = (fhiy - Py) * iy;
-                const float z1 = (floz - Pz) * iz, z2 = (fhiz - Pz) * iz;
-                const float nrx = fminf(x1, x2), nry = fminf(y1, y2), nrz = fminf(z1, z2);
-                const float tn = max3f(nrx, nry, nrz);
-                const float tf = min3f(fmaxf(x1, x2), fmaxf(y1, y2), fmaxf(z1, z2));
-                const bool alive = any_voxel && (tn <= tf) && (tf > 0.0f);
-                const int eaxis = tn < 0.0f ? -1 : (nrx == tn ? 0 : (nry == tn ? 1 : 2));
-                t_hit = alive ? fmaxf(tn, 0.0f) : 0.0f;
-                int cx = min(max((int)floorf(fmaf(t_hit, dx, Px)), lox), hix - 1);
-                int cy = min(max((int)floorf(fmaf(t_hit, dy, Py)), loy), hiy - 1);
-                int cz = min(max((int)floorf(fmaf(t_hit, dz, Pz)), loz), hiz - 1);
-                if (eaxis == 0) cx = ngx ? hix - 1 : lox;
-                if (eaxis == 1) cy = ngy ? hiy - 1 : loy;
-                if (eaxis == 2) cz = ngz ? hiz - 1 : loz;
-                if (!alive) { cx = cy = cz = 0; }
-                const int v = stride_x * cx + stride_z * cz + stride_y * cy;
-                vi = (uint32_t)v + vi_bias;
-                t0x = ((float)(cx + (ngx ? 0 : 1)) - Px) * ix;
-                t0y = ((float)(cy + (ngy ? 0 : 1)) - Py) * iy;
-                t0z = ((float)(cz + (ngz ? 0 : 1)) - Pz) * iz;
-                t_exit = min3f(fmaf(ngx ? (float)(cx - lox) : (float)(hix - 1 - cx), dtx, t0x),
-                               fmaf(ngy ? (float)(cy - loy) : (float)(hiy - 1 - cy), dty, t0y),
-                               fmaf(ngz ? (float)(cz - loz) : (float)(hiz - 1 - cz), dtz, t0z)) * p.exit_scale;
-                const bool filled = alive && ((s_occ[v >> 5] >> (v & 31)) & 1u);
-                // entered through the box face of axis eaxis, or the eye is inside a solid
-                if (filled) row = eaxis < 0 ? inside_row : face_row(eaxis);
-                if (!alive || filled) t_exit = -kInf;
-            }
+            uint32_t pos, bit = 0, row, sgn3;
+            float t_hit, dtx, dty, dtz;
+            if (COLW && cam_in) {
+                // ---- the common case in one block of PTX: tile record, ray through the pixel centre
+                // (d = F + a*Rs + b*Us, a = 2px+1-W, b = H-1-2py, two chained FMAs per component; a
+                // component that is exactly zero becomes 1e-30 so that it never crosses a cell face and
+                // the slab arithmetic stays finite), reciprocals, the DDA table rows for the ray's signs
+                // {distance to the first face, cells left, step, colour row} per axis, first crossing
+                // times, exit time, then the walk.  The basis is re-read from shared memory per tile:
+                // three broadcast loads cost less than nine registers held across the walk.
+                asm volatile("{\n"
+                    MV_DDA_DECL
+                    " .reg .f32 Ta, Tb, Fx, Fy, Fz, Rx, Ry, Rz, Ux, Uy, Uz, ca, cb, dx, dy, dz, ix, iy, iz;\n"
+                    " .reg .f32 q0, q1, q2, q3, q4, q5, esc;\n"
+                    " .reg .b32 u, tab;\n"
+                    " .reg .pred p0;\n"
+                    " ld.shared.v4.b32 {Ta, Tb, %0, _}, [%9];\n"
+                    " ld.shared.f32 Fx, [%10+12];\n"
+                    " ld.shared.v4.f32 {Fy, Fz, Rx, Ry}, [%10+16];\n"
+                    " ld.shared.v4.f32 {Rz, Ux, Uy, Uz}, [%10+32];\n"
+                    " ld.shared.v4.b32 {bit, esc, %4, pos}, [%10+64];\n"
+                    " add.f32 ca, Ta, %11;\n"
+                    " sub.f32 cb, Tb, %12;\n"
+                    " fma.rn.f32 dx, ca, Rx, Fx;\n"
+                    " fma.rn.f32 dy, ca, Ry, Fy;\n"
+                    " fma.rn.f32 dz, ca, Rz, Fz;\n"
+                    " fma.rn.f32 dx, cb, Ux, dx;\n"
+                    " fma.rn.f32 dy, cb, Uy, dy;\n"
+                    " fma.rn.f32 dz, cb, Uz, dz;\n"
+                    " setp.eq.f32 p0, dx, 0f00000000;\n"
+                    " selp.f32 dx, 0f0DA24260, dx, p0;\n"
+                    " setp.eq.f32 p0, dy, 0f00000000;\n"
+                    " selp.f32 dy, 0f0DA24260, dy, p0;\n"
+                    " setp.eq.f32 p0, dz, 0f00000000;\n"
+                    " selp.f32 dz, 0f0DA24260, dz, p0;\n"
+                    " rcp.approx.ftz.f32 ix, dx;\n"
+                    " rcp.approx.ftz.f32 iy, dy;\n"
+                    " rcp.approx.ftz.f32 iz, dz;\n"
+                    " abs.f32 dtx, ix;\n"
+                    " abs.f32 dty, iy;\n"
+                    " abs.f32 dtz, iz;\n"
+                    " mov.b32 u, dx;\n"
+                    " shr.u32 %8, u, 31;\n"
+                    " mov.b32 u, dy;\n"
+                    " shr.u32 u, u, 30;\n"
+                    " lop3.b32 %8, u, 2, %8, 0xEA;\n"
+                    " mov.b32 u, dz;\n"
+                    " shr.u32 u, u, 29;\n"
+                    " lop3.b32 %8, u, 4, %8, 0xEA;\n"
+                    " mad.lo.u32 tab, %8, 48, %10;\n"
+                    " ld.shared.v4.b32 {q0, q1, sx, _}, [tab+" MV_TAB_X "];\n"
+                    " ld.shared.v4.b32 {q2, q3, sy, _}, [tab+" MV_TAB_Y "];\n"
+                    " ld.shared.v4.b32 {q4, q5, sz, _}, [tab+" MV_TAB_Z "];\n"
+                    " mul.f32 tx, q0, ix;\n"
+                    " mul.f32 ty, q2, iy;\n"
+                    " mul.f32 tz, q4, iz;\n"
+                    " fma.rn.f32 q1, q1, dtx, tx;\n"
+                    " fma.rn.f32 q3, q3, dty, ty;\n"
+                    " fma.rn.f32 q5, q5, dtz, tz;\n"
+                    " min.f32 q1, q1, q3, q5;\n"
+                    " mul.f32 texit, q1, esc;\n"
 #if MV_PROBE >= 1 && MV_PROBE < 9
-            t_exit = -kInf;
+                    " mov.f32 texit, 0fFF800000;\n"
 #endif
-            // The crossing times accumulate (t += dt), so after n steps they differ from the exact
-            // products by up to n roundings; the exit time was pulled in by that bound, which keeps
-            // the walk inside the box.
-            // 3D-DDA written in PTX so that each step is a fixed short sequence of predicated
-            // instructions (see MV_DDA_ADVANCE); four steps per trip of the bounded loop.
-            {
-                const int budget = p.max_steps;
-                if constexpr (OCC_SHARED) {
-                    asm volatile(MV_DDA_BODY
-                                 : "+r"(vi), "+f"(t_hit), "+r"(row), "+f"(t0x), "+f"(t0y), "+f"(t0z)
-                                 : "f"(dtx), "f"(dty), "f"(dtz), "r"(sx), "r"(sy), "r"(sz), "f"(t_exit), "r"(budget),
-                                   "r"(tab), "l"(0ull)
-                                 : "memory");
+                    " mov.f32 thit, 0f00000000;\n"
+                    " mov.s32 it, " MV_STEP_BUDGET ";\n"
+                    MV_DDA_LOOP(MV_DDA_STEP_COLW)
+                    " selp.u32 a, 16, 32, py;\n"
+                    " selp.u32 a, 0, a, px;\n"
+                    " add.u32 a, a, tab;\n"
+                    " @ph ld.shared.u32 %4, [a+" MV_TAB_ROW "];\n"
+#if MV_PROBE == 9
+                    " mov.f32 thit, ns;\n"
+#endif
+                    " mov.b32 %1, pos;\n"
+                    " mov.b32 %2, bit;\n"
+                    " mov.f32 %3, thit;\n"
+                    " mov.f32 %5, dtx;\n"
+                    " mov.f32 %6, dty;\n"
+                    " mov.f32 %7, dtz;\n"
+                    "}\n"
+                    : "=&r"(tile_px), "=&r"(pos), "=&r"(bit), "=&f"(t_hit), "=&r"(row), "=&f"(dtx), "=&f"(dty), "=&f"(dtz), "=&r"(sgn3)
+                    : "r"(tile_p), "r"(abase), "f"(lane_a), "f"(lane_b)
+                    : "memory");
+            } else {
+                // ---- every other case: the same steps in C++, with the eye possibly outside the
+                // occupied box and either flavour of the walk
+                float Ta, Tb;
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, _}, [%3];" : "=f"(Ta), "=f"(Tb), "=r"(tile_px) : "r"(tile_p));
+                float Fx, Fy, Fz, Rx, Ry, Rz, Ux, Uy, Uz, esc;
+                uint32_t pos0, row0, bit0;
+                asm volatile("ld.shared.f32 %0, [%1+12];" : "=f"(Fx) : "r"(abase));
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4+16];" : "=f"(Fy), "=f"(Fz), "=f"(Rx), "=f"(Ry) : "r"(abase));
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4+32];" : "=f"(Rz), "=f"(Ux), "=f"(Uy), "=f"(Uz) : "r"(abase));
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4+64];" : "=r"(bit0), "=f"(esc), "=r"(row0), "=r"(pos0) : "r"(abase));
+                const float a = Ta + lane_a, bb = Tb - lane_b;
+                float dx = fmaf(bb, Ux, fmaf(a, Rx, Fx));
+                float dy = fmaf(bb, Uy, fmaf(a, Ry, Fy));
+                float dz = fmaf(bb, Uz, fmaf(a, Rz, Fz));
+                dx = dx == 0.0f ? 1e-30f : dx;
+                dy = dy == 0.0f ? 1e-30f : dy;
+                dz = dz == 0.0f ? 1e-30f : dz;
+                const float ix = fast_rcp(dx), iy = fast_rcp(dy), iz = fast_rcp(dz);
+                dtx = fabsf(ix); dty = fabsf(iy); dtz = fabsf(iz);
+                sgn3 = (__float_as_uint(dx) >> 31) | ((__float_as_uint(dy) >> 30) & 2u) | ((__float_as_uint(dz) >> 29) & 4u);
+                const uint32_t tab = abase + 48u * sgn3;
+                float qxx, qxy, qyx, qyy, qzx, qzy;
+                int sx, sy, sz;
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, _}, [%3+" MV_TAB_X "];" : "=f"(qxx), "=f"(qxy), "=r"(sx) : "r"(tab));
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, _}, [%3+" MV_TAB_Y "];" : "=f"(qyx), "=f"(qyy), "=r"(sy) : "r"(tab));
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, _}, [%3+" MV_TAB_Z "];" : "=f"(qzx), "=f"(qzy), "=r"(sz) : "r"(tab));
+                float t0x, t0y, t0z, t_exit;
+                t_hit = 0.0f;
+                pos = pos0; bit = bit0; row = row0;
+                if (cam_in) {
+                    t0x = qxx * ix;
+                    t0y = qyx * iy;
+                    t0z = qzx * iz;
+                    t_exit = min3f(fmaf(qxy, dtx, t0x), fmaf(qyy, dty, t0y), fmaf(qzy, dtz, t0z)) * esc;
                 } else {
-                    asm volatile(MV_DDA_BODY_GLOBAL
-                                 : "+r"(vi), "+f"(t_hit), "+r"(row), "+f"(t0x), "+f"(t0y), "+f"(t0z)
-                                 : "f"(dtx), "f"(dty), "f"(dtz), "r"(sx), "r"(sy), "r"(sz), "f"(t_exit), "r"(budget),
-                                   "r"(tab), "l"(s_occ)
-                                 : "memory");
+                    // eye outside the occupied box: clip the ray to it, start in the entry cell
+                    const bool ngx = dx < 0.0f, ngy = dy < 0.0f, ngz = dz < 0.0f;
+                    const float x1 = (flox - Px) * ix, x2 = (fhix - Px) * ix;
+                    const float y1 = (floy - Py) * iy, y2 = (fhiy - Py) * iy;
+                    const float z1 = (floz - Pz) * iz, z2 = (fhiz - Pz) * iz;
+                    const float nrx = fminf(x1, x2), nry = fminf(y1, y2), nrz = fminf(z1, z2);
+                    const float tn = max3f(nrx, nry, nrz);
+                    const float tf = min3f(fmaxf(x1, x2), fmaxf(y1, y2), fmaxf(z1, z2));
+                    const bool alive = any_voxel && (tn <= tf) && (tf > 0.0f);
+                    const int eaxis = tn < 0.0f ? -1 : (nrx == tn ? 0 : (nry == tn ? 1 : 2));
+                    t_hit = alive ? fmaxf(tn, 0.0f) : 0.0f;
+                    int cx = min(max((int)floorf(fmaf(t_hit, dx, Px)), lox), hix - 1);
+                    int cy = min(max((int)floorf(fmaf(t_hit, dy, Py)), loy), hiy - 1);
+                    int cz = min(max((int)floorf(fmaf(t_hit, dz, Pz)), loz), hiz - 1);
+                    if (eaxis == 0) cx = ngx ? hix - 1 : lox;
+                    if (eaxis == 1) cy = ngy ? hiy - 1 : loy;
+                    if (eaxis == 2) cz = ngz ? hiz - 1 : loz;
+                    if (!alive) { cx = cy = cz = 0; }
+                    pos = cell_pos(cx, cy, cz);
+                    bit = 1u << cy;
+                    t0x = ((float)(cx + (ngx ? 0 : 1)) - Px) * ix;
+                    t0y = ((float)(cy + (ngy ? 0 : 1)) - Py) * iy;
+                    t0z = ((float)(cz + (ngz ? 0 : 1)) - Pz) * iz;
+                    t_exit = min3f(fmaf(ngx ? (float)(cx - lox) : (float)(hix - 1 - cx), dtx, t0x),
+                                   fmaf(ngy ? (float)(cy - loy) : (float)(hiy - 1 - cy), dty, t0y),
+                                   fmaf(ngz ? (float)(cz - loz) : (float)(hiz - 1 - cz), dtz, t0z)) * p.exit_scale;
+                    const bool filled = alive && cell_filled(cx, cy, cz);
+                    // entered through the box face of axis eaxis, or the eye is inside a solid
+                    if (filled) {
+                        if (eaxis < 0) row = inside_row;
+                        else asm volatile("ld.shared.u32 %0, [%1+" MV_TAB_ROW "];" : "=r"(row) : "r"(tab + 16u * (uint32_t)eaxis));
+                    }
+                    if (!alive || filled) t_exit = -kInf;
                 }
+#if MV_PROBE >= 1 && MV_PROBE < 9
+                t_exit = -kInf;
+#endif
+#define MV_DDA_IO                                                                                         \
+                    : "+r"(pos), "+r"(bit), "+f"(t_hit), "+r"(row)                                                  \
+                    : "f"(t0x), "f"(t0y), "f"(t0z), "f"(dtx), "f"(dty), "f"(dtz), "r"(sx), "r"(sy), "r"(sz), "f"(t_exit), \
+                      "r"(p.max_steps), "r"(tab), "l"(s_occ)                                                       \
+                    : "memory"
+#define MV_DDA_IN                                                                                         \
+                    " mov.b32 pos, %0;\n mov.b32 bit, %1;\n mov.f32 thit, %2;\n"                                    \
+                    " mov.f32 tx, %4;\n mov.f32 ty, %5;\n mov.f32 tz, %6;\n mov.f32 dtx, %7;\n mov.f32 dty, %8;\n"   \
+                    " mov.f32 dtz, %9;\n mov.b32 sx, %10;\n mov.b32 sy, %11;\n mov.b32 sz, %12;\n mov.f32 texit, %13;\n" \
+                    " mov.s32 it, " MV_STEP_BUDGET ";\n mov.b64 gbase, %16;\n"
+#define MV_DDA_OUTS                                                                                       \
+                    " selp.u32 a, 16, 32, py;\n selp.u32 a, 0, a, px;\n add.u32 a, a, %15;\n"                        \
+                    " @ph ld.shared.u32 %3, [a+" MV_TAB_ROW "];\n mov.b32 %0, pos;\n mov.b32 %1, bit;\n mov.f32 %2, thit;\n"
+                if constexpr (COLW) {
+                    asm volatile("{\n" MV_DDA_DECL MV_DDA_IN MV_DDA_LOOP(MV_DDA_STEP_COLW) MV_DDA_OUTS "}\n" MV_DDA_IO);
+                } else if constexpr (OCC_SHARED) {
+                    asm volatile("{\n" MV_DDA_DECL MV_DDA_IN MV_DDA_LOOP(MV_DDA_STEP_IDX) MV_DDA_OUTS "}\n" MV_DDA_IO);
+                } else {
+                    asm volatile("{\n" MV_DDA_DECL MV_DDA_IN MV_DDA_LOOP(MV_DDA_STEP_IDX_GLOBAL) MV_DDA_OUTS "}\n" MV_DDA_IO);
+                }
+#undef MV_DDA_IO
+#undef MV_DDA_IN
+#undef MV_DDA_OUTS
             }
             __syncwarp();
-            const bool vhit = row != kNoRow;
 
-            // ---- voxel colour: one material byte from global memory, then the shaded table
-            uint32_t rgbx = p.sky_rgbx;
-            float depth = p.miss_depth;
-            if (vhit) {
-                const uint32_t m = __ldg(mat_lane + vi);
-                asm("ld.shared.u32 %0, [%1];" : "=r"(rgbx) : "r"(row + 4u * m));
-                depth = t_hit;
+            // ---- voxel colour (one material byte from global memory, then the shaded table), this
+            // tile's first box-mask word, and the latest voxel hit of the warp (boxes wholly behind it
+            // are skipped).  Predicated, not branched; sky colour and miss depth ride with the material
+            // store's address in the agent block.  (Column-word flavour: the voxel index is rebuilt from
+            // the column's address and the bit.)
+            uint32_t rgbx, m;
+            float depth, tb, wmax;
+            {
+                const uint32_t vi = COLW ? (pos << 3) + (uint32_t)(31 - __clz(bit)) : pos;
+                asm volatile("{\n"
+                    " .reg .pred pv;\n"
+                    " .reg .b32 mid, skyb, missb, tbb, wmb;\n"
+                    " .reg .b64 mp, sm;\n"
+                    " ld.shared.v2.b64 {mp, sm}, [%8+80];\n"
+                    " ld.shared.u32 %2, [%9];\n"
+                    " mov.b64 {skyb, missb}, sm;\n"
+                    " mov.b32 %0, skyb;\n"
+                    " mov.b32 %1, missb;\n"
+                    " setp.ne.u32 pv, %5, 0xffffffff;\n"
+                    " cvt.u64.u32 sm, %6;\n"
+                    " add.u64 mp, mp, sm;\n"
+                    " mov.b32 tbb, 0x7F800000;\n"
+                    " @pv ld.global.nc.u8 mid, [mp];\n"
+                    " @pv mov.b32 tbb, %7;\n"
+                    " @pv mad.lo.u32 mid, mid, 4, %5;\n"
+                    " redux.sync.max.u32 wmb, tbb, 0xffffffff;\n"
+                    " mov.b32 %3, tbb;\n"
+                    " mov.b32 %4, wmb;\n"
+                    " @pv ld.shared.u32 %0, [mid];\n"
+                    " @pv mov.f32 %1, %7;\n"
+                    "}\n"
+                    : "=&r"(rgbx), "=&f"(depth), "=&r"(m), "=&f"(tb), "=&f"(wmax)
+                    : "r"(row), "r"(vi), "f"(t_hit), "r"(abase), "r"(mask_p)
+                    : "memory");
             }
 #if MV_PROBE == 9
             depth = t_hit;
 #endif
-
-            // ---- boxes of this tile (skip those wholly behind every lane's voxel hit); a box wins
-            // only with a strictly smaller time
-            {
-                uint32_t m;
-                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(m) : "r"(mask_p));
 #if MV_PROBE >= 2 && MV_PROBE < 9
-                m = 0;
+            m = 0;
 #endif
-                float tb = vhit ? t_hit : kInf;
-                const float wmax = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(tb)));
+
+            // ---- boxes of this tile; a box wins only with a strictly smaller time
+            {
                 if (m != 0u || mw > 1) {
-                    // signed reciprocals again: the index strides carry the signs of the direction
-                    const float ix = __uint_as_float(__float_as_uint(dtx) | ((uint32_t)sx & 0x80000000u));
-                    const float iy = __uint_as_float(__float_as_uint(dty) | ((uint32_t)sy & 0x80000000u));
-                    const float iz = __uint_as_float(__float_as_uint(dtz) | ((uint32_t)sz & 0x80000000u));
+                    // signed reciprocals again, and the ray's rows of the DDA table for the faces
+                    const float ix = __uint_as_float(__float_as_uint(dtx) | (sgn3 << 31));
+                    const float iy = __uint_as_float(__float_as_uint(dty) | ((sgn3 & 2u) << 30));
+                    const float iz = __uint_as_float(__float_as_uint(dtz) | ((sgn3 & 4u) << 29));
+                    const uint32_t tab = abase + 48u * sgn3;
                     uint32_t baddr = 0;
                     for (int w = 0;;) {
                         while (m) {
                             const int b = (__ffs(m) - 1) + 32 * w;
                             m &= m - 1;
-                            const float4 lo = rel[2 * b], hi = rel[2 * b + 1];
+                            float4 lo, hi;
+                            const uint32_t rel_p = abase + kAgentRelOff + 32u * (uint32_t)b;
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(lo.x), "=f"(lo.y), "=f"(lo.z), "=f"(lo.w) : "r"(rel_p));
                             if (lo.w > wmax) continue;
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4+16];" : "=f"(hi.x), "=f"(hi.y), "=f"(hi.z), "=f"(hi.w) : "r"(rel_p));
                             const float x1 = lo.x * ix, x2 = hi.x * ix, y1 = lo.y * iy, y2 = hi.y * iy;
                             const float z1 = lo.z * iz, z2 = hi.z * iz;
                             const float nx = fminf(x1, x2), ny = fminf(y1, y2), nz = fminf(z1, z2);
@@ -561,7 +702,10 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                             const float t = fmaxf(tn, 0.0f);
                             if ((tn <= tf) && (tf > 0.0f) && (t < tb)) {
                                 tb = t;
-                                const uint32_t r = (tn < 0.0f) ? inside_row : face_row((nx == tn) ? 0 : ((ny == tn) ? 1 : 2));
+                                uint32_t r = inside_row;
+                                if (!(tn < 0.0f))
+                                    asm volatile("ld.shared.u32 %0, [%1+" MV_TAB_ROW "];" : "=r"(r)
+                                                 : "r"(tab + ((nx == tn) ? 0u : ((ny == tn) ? 16u : 32u))));
                                 baddr = r + 4u * __float_as_uint(hi.w);
                             }
                         }
@@ -576,22 +720,35 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             }
 
             // ---- GUI overlay: rectangles in list order, later ones on top; depth is left alone
-            if (ov_count > 0 && ((ovtile[tile_no >> 5] >> (tile_no & 31)) & 1u)) {
-                const int px = (tile_px % W) + (lane & 7), py = (tile_px / W) + (lane >> 3);
-                for (int r = 0; r < ov_count; ++r) {
-                    const int4 q = ov[2 * r];
-                    if (px >= q.x && px < q.z && py >= q.y && py < q.w) rgbx = (uint32_t)ov[2 * r + 1].x;
+            if (ov_count > 0) {
+                const uint32_t tile_no = (tile_p - smem_addr(s_tile)) >> 4;
+                if ((agent_ovtile(ag)[tile_no >> 5] >> (tile_no & 31)) & 1u) {
+                    const int4 *ov = agent_ov(ag);
+                    const int px = (tile_px % W) + (lane & 7), py = (tile_px / W) + (lane >> 3);
+                    for (int r = 0; r < ov_count; ++r) {
+                        const int4 q = ov[2 * r];
+                        if (px >= q.x && px < q.z && py >= q.y && py < q.w) rgbx = (uint32_t)ov[2 * r + 1].x;
+                    }
                 }
             }
 
             // ---- store: depth rows are 32-byte segments; RGB rows are 24 bytes = 6 packed words
-            depth_lane[tile_px] = depth;
-            {
-                const uint32_t ca = __shfl_sync(0xffffffffu, rgbx, st_src);
-                const uint32_t cb = __shfl_sync(0xffffffffu, rgbx, st_src + 1);
-                const uint32_t word = __byte_perm(ca, cb, st_sel);
-                if ((int)st_sel >= 0) *reinterpret_cast<uint32_t *>(rgb_lane + 3 * tile_px) = word;
-            }
+            asm volatile("{\n"
+                " .reg .pred ps;\n"
+                " .reg .b32 ca, cb, s2;\n"
+                " .reg .b64 ad;\n"
+                " mad.wide.s32 ad, %2, 4, %3;\n"
+                " st.global.f32 [ad], %1;\n"
+                " shfl.sync.idx.b32 ca, %0, %5, 31, 0xffffffff;\n"
+                " add.u32 s2, %5, 1;\n"
+                " shfl.sync.idx.b32 cb, %0, s2, 31, 0xffffffff;\n"
+                " mad.wide.s32 ad, %2, 3, %4;\n"
+                " prmt.b32 ca, ca, cb, %6;\n"
+                " setp.ge.s32 ps, %6, 0;\n"
+                " @ps st.global.u32 [ad], ca;\n"
+                "}\n"
+                :: "r"(rgbx), "f"(depth), "r"(tile_px), "l"(depth_lane), "l"(rgb_lane), "r"(st_src), "r"(st_sel)
+                : "memory");
         }
     }
 }
