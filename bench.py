@@ -7,9 +7,13 @@
 A step is one pass of the whole per-step path: mv_set_cameras + mv_render_batch over the whole
 batch, inputs resident in HBM.  `value` is observations per second over all ranks (device time,
 CUDA events, max over ranks); `e2e` is the same metric through mv_step_host with page-locked host
-buffers (cameras and boxes copied in, frames copied out, every step).  With N > 1 (torchrun) every
-rank renders its own 16384 seeded environments: no data-path collective (weak scaling).
-`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+buffers (cameras and boxes copied in, frames copied out, every step).  With --gpus N > 1 the script
+starts N ranks itself (one per GPU, through torch.distributed.run) unless it already runs under
+such a launcher; every rank renders its own 16384 seeded environments and nothing is exchanged on
+the data path (weak scaling).  `--plan` prints which rank renders which environments and touches
+no GPU.  `--impl reference` times the CPU oracle on a bounded sample of the same workload.
+The sweep workload (`--workload sweep`) precedes every step by its seeded camera update, the
+sequences pre-computed on the device.
 """
 from __future__ import annotations
 
@@ -27,12 +31,14 @@ ROOT = Path(__file__).resolve().parent
 sys.path.insert(0, str(ROOT))
 
 WORKLOAD = "headline"
-# DRAM bytes (read 1.24 GB + write 1.01 GB) of one render_kernel launch on this full workload, from
-# the one-pass ncu capture summarised in profiles/render_kernel_headline_launch_list.md.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 2.25e9
-# Warp instructions the render kernel executes per 8x4-pixel tile on this workload
-# (smsp__inst_executed.sum / tiles, profiles/render_kernel_headline_2048env_ncu_full.md).
-NCU_WARP_INSTRUCTIONS_PER_TILE = 435
+# Profiler evidence that the bench line quotes next to its live timings.  Both figures come from one ncu
+# capture of render_kernel on a 2048-environment slice of the headline workload (summary and command in
+# profiles/render_kernel_headline_2048env_ncu.md); NCU_BUILD names the commit of the library they were
+# taken on.  DRAM traffic grows in proportion to the environments, so a full launch is the slice x 8.
+NCU_BUILD = "unset"
+NCU_SLICE_ENVS = 2048
+NCU_SLICE_DRAM_BYTES = None          # dram__bytes_read.sum + dram__bytes_write.sum of one launch on the slice
+NCU_WARP_INSTRUCTIONS_PER_TILE = None  # smsp__inst_executed.sum / (8x4-pixel tiles) on the slice
 
 
 def measured_peak():
@@ -102,6 +108,19 @@ class ClockSampler:
             return {"sm_mhz": a, "sm_max_mhz": b, "samples": 1, "reasons": ["sampled after the timed region (NVML unavailable)"]}
         except Exception:               # noqa: BLE001
             return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["clock sampling unavailable"]}
+
+
+def cpu_affinity() -> str:
+    """The cores this process may run on, as a compact range list."""
+    cores = sorted(os.sched_getaffinity(0))
+    out, i = [], 0
+    while i < len(cores):
+        j = i
+        while j + 1 < len(cores) and cores[j + 1] == cores[j] + 1:
+            j += 1
+        out.append(str(cores[i]) if i == j else f"{cores[i]}-{cores[j]}")
+        i = j + 1
+    return ",".join(out)
 
 
 def cpu_model() -> str:
@@ -204,9 +223,29 @@ def run_reference(args, rank):
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": workload_config(cfg, args.gpus),
         "cpu_baseline": {"value": value, "unit": "obs/s", "cores": cores, "kind": "oracle", "cpu_model": cpu_model(),
-                         "sample": what},
+                         "affinity": cpu_affinity(), "sample": what},
         "e2e": {"value": value, "unit": "obs/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+def run_plan(args, rank, world):
+    """Rank -> seeded environment range, gathered over the same launcher as the benchmark but on the
+    CPU backend: every rank reports its own range, rank 0 prints them.  No CUDA call is made."""
+    from paper_2107_08170_b200 import scenes, shard
+    over = {"num_envs": args.envs} if args.envs is not None else {}
+    cfg = scenes.config(WORKLOAD, **over)
+    begin = shard.env_offset(rank, cfg.num_envs)
+    mine = {"rank": rank, "env_begin": begin, "env_end": begin + cfg.num_envs, "observations": cfg.num_obs}
+    plan = [mine]
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("gloo")
+        plan = [None] * world
+        dist.all_gather_object(plan, mine)
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"plan": plan, "n_gpus": world, "workload": WORKLOAD, "scaling": "weak",
+                          "collectives_on_data_path": 0}))
 
 
 def workload_config(cfg, n_gpus):
@@ -236,8 +275,16 @@ def main():
     ap.add_argument("--height", type=int, default=None)
     ap.add_argument("--extras", action="store_true",
                     help="also time the overlay, agent-motion and voxel-merge entry points (adds an \"extras\" object)")
+    ap.add_argument("--plan", action="store_true",
+                    help="print which rank renders which seeded environments and exit (no GPU is touched)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" and args.envs is None else args.warmup
+
+    # --gpus N on its own starts the N ranks (one per GPU); under a launcher the ranks are already there
+    if args.gpus > 1 and "RANK" not in os.environ and not (args.impl == "reference"):
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--standalone", "--local-addr", "127.0.0.1", "--nnodes=1",
+               f"--nproc-per-node={args.gpus}", str(Path(__file__).resolve()), *sys.argv[1:]]
+        raise SystemExit(subprocess.call(cmd))
 
     global WORKLOAD
     WORKLOAD = args.workload
@@ -246,6 +293,9 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", 0))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.plan:
+        run_plan(args, rank, world)
         return
 
     import torch
@@ -272,8 +322,13 @@ def main():
     step_bytes = workload.algorithmic_bytes(cfg)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if step_bytes < (512 << 20) else None
     keep = list(range(0, cfg.num_envs, max(cfg.num_envs // 8, 1)))[:8] if rank == 0 and not args.no_cpu else []
+    # the sweep workload moves every camera before every step (seeded walk, pre-computed here)
+    walk_steps = args.steps + args.warmup if WORKLOAD == "sweep" else 0
     batch, cams, kept = workload.build_batch(cfg, local, env_offset=shard.env_offset(rank, cfg.num_envs), keep_envs=keep,
-                                             max_overlay_rects=1 if args.extras else 0)
+                                             max_overlay_rects=1 if args.extras else 0, camera_walk_steps=walk_steps)
+    cam_seq = cams[1:] if walk_steps else None
+    if walk_steps:
+        cams = cams[0]
     rgb, depth = batch.alloc_outputs()
     stream = torch.cuda.current_stream()
 
@@ -282,12 +337,12 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    def step():
-        batch.set_cameras(cams)
+    def step(i):
+        batch.set_cameras(cam_seq[i] if cam_seq is not None else cams)
         batch.render_batch(rgb, depth)
 
-    for _ in range(args.warmup):
-        step()
+    for i in range(args.warmup):
+        step(i)
     barrier()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -296,11 +351,11 @@ def main():
     launches0 = batch.launch_count()
     barrier()
     t_begin.record(stream)
-    for e0, e1, e2 in ev:
+    for i, (e0, e1, e2) in enumerate(ev):
         if flush is not None:
             flush.fill_(1)
         e0.record(stream)
-        batch.set_cameras(cams)
+        batch.set_cameras(cam_seq[args.warmup + i] if cam_seq is not None else cams)
         e1.record(stream)
         batch.render_batch(rgb, depth)
         e2.record(stream)
@@ -361,9 +416,9 @@ def main():
         alg = workload.algorithmic_bytes(cfg)
         k_ms = statistics.mean(render_ms)
         achieved = alg / (k_ms * 1e-3) / 1e9
-        traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH if WORKLOAD == "headline" else None
-        if traffic is not None and args.envs is not None:
-            traffic = traffic * cfg.num_envs / 16384
+        traffic = None
+        if WORKLOAD == "headline" and NCU_SLICE_DRAM_BYTES is not None:       # scaled from the profiled slice
+            traffic = NCU_SLICE_DRAM_BYTES * cfg.num_envs / NCU_SLICE_ENVS
         out = {
             "metric": "observations/sec", "value": value, "unit": "obs/s",
             "grays_per_sec": value * px / 1e9,
@@ -373,17 +428,20 @@ def main():
             "clocks": clocks, "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "kernel": "render_kernel", "achieved": achieved, "peak": peak,
                          "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": traffic, "algorithmic_bytes_per_launch": alg,
+                         "traffic": traffic, "traffic_build": NCU_BUILD,
+                         "traffic_how": f"ncu dram bytes of one launch on a {NCU_SLICE_ENVS}-env slice, scaled by envs",
+                         "algorithmic_bytes_per_launch": alg,
                          "kernel_ms_mean": k_ms, "kernel_ms_min": min(render_ms), "kernel_ms_median": statistics.median(render_ms)},
             # the resource that actually binds: warp-instruction issue slots (one per scheduler per cycle)
-            "issue_roofline": {"bound": "alu", "unit": "warp-instructions/s",
-                               "achieved": NCU_WARP_INSTRUCTIONS_PER_TILE * (cfg.num_obs * px / 32) / (k_ms * 1e-3),
+            "issue_roofline": {"bound": "alu", "unit": "warp-instructions/s", "counter_build": NCU_BUILD,
+                               "warp_instructions_per_tile": NCU_WARP_INSTRUCTIONS_PER_TILE,
+                               "achieved": (NCU_WARP_INSTRUCTIONS_PER_TILE or 0) * (cfg.num_obs * px / 32) / (k_ms * 1e-3),
                                "peak": 148 * 4 * (clocks.get("sm_mhz") or 1965.0) * 1e6,
                                "peak_kind": "148 SMs x 4 schedulers x sampled SM clock"},
             "paper_context": "paper: 1.1e6 obs/s whole simulator on one 8x RTX 2080 Ti node (128x72 RGB, no depth)",
         }
         out["issue_roofline"]["frac"] = out["issue_roofline"]["achieved"] / out["issue_roofline"]["peak"]
-        if WORKLOAD != "headline":                 # the instructions-per-tile figure was measured on the headline workload
+        if WORKLOAD != "headline" or NCU_WARP_INSTRUCTIONS_PER_TILE is None:   # the figure belongs to the headline workload
             out.pop("issue_roofline")
         if e2e:
             out["e2e"] = {"value": obs_total / (e2e[0] * 1e-3), "unit": "obs/s", "ms_per_step": e2e[0],
@@ -391,6 +449,7 @@ def main():
         if not args.no_cpu and kept:
             rate, n, secs, cores = cpu_oracle_rate(cfg, kept)
             out["cpu_baseline"] = {"value": rate, "unit": "obs/s", "cores": cores, "kind": "oracle", "cpu_model": cpu_model(),
+                                   "affinity": cpu_affinity(),
                                    "sample": f"{n} observations (every {max(cfg.num_envs // 8, 1)}th env) of this workload, all pixels, {secs:.1f} s"}
         print(json.dumps(out))
     if args.extras and rank == 0:

@@ -18,12 +18,15 @@ def algorithmic_bytes(cfg) -> int:
 
 
 def build_batch(cfg, device: int = 0, env_offset: int = 0, keep_envs=(), chunk_envs: int = 512,
-                max_overlay_rects: int = 0):
+                max_overlay_rects: int = 0, camera_walk_steps: int = 0):
     """Returns (batch, cams_dev, kept) where kept[e] holds CPU arrays of env e (local index)
-    for every e in keep_envs.  env_offset shifts the seeded env ids (one range per rank)."""
+    for every e in keep_envs.  env_offset shifts the seeded env ids (one range per rank).
+    With camera_walk_steps = K the second element is a list of K+1 camera tensors: the initial cameras
+    followed by K seeded updates of the sweep workload (scenes.walk_cameras), pre-computed on the device."""
     dev = torch.device("cuda", device)
     batch = binding.Batch(binding.desc_from_config(cfg, device, max_overlay_rects))
     cams = torch.empty(cfg.num_obs, 6, dtype=torch.int32, device=dev)
+    walk = [torch.empty_like(cams) for _ in range(camera_walk_steps)]
     kept = {}
     keep = set(int(e) for e in keep_envs)
     A = cfg.agents
@@ -35,6 +38,10 @@ def build_batch(cfg, device: int = 0, env_offset: int = 0, keep_envs=(), chunk_e
             boxes, count = sc["boxes"].contiguous(), sc["box_count"].contiguous()
         batch.upload_worlds(e0, n, sc["grid"].contiguous(), boxes, count, sc["palette"].contiguous())
         cams[e0 * A:(e0 + n) * A] = sc["cams"]
+        step_cams = sc["cams"]
+        for k in range(camera_walk_steps):
+            step_cams = scenes.walk_cameras(cfg, sc, step_cams, k + 1)
+            walk[k][e0 * A:(e0 + n) * A] = step_cams
         for e in keep:
             if e0 <= e < e0 + n:
                 i = e - e0
@@ -43,4 +50,4 @@ def build_batch(cfg, device: int = 0, env_offset: int = 0, keep_envs=(), chunk_e
                            "cams": sc["cams"][i * A:(i + 1) * A].cpu().numpy()}
         torch.cuda.synchronize(dev)
         del sc
-    return batch, cams, kept
+    return batch, ([cams] + walk if camera_walk_steps else cams), kept

@@ -87,8 +87,12 @@ def test_move_agents_matches_oracle_then_renders(oracle):
             boxes[e, sb, :3] = lo.astype(np.float32).view(np.int32)
             boxes[e, sb, 3:6] = hi.astype(np.float32).view(np.int32)
         g = d_cams.cpu().numpy()
-        mismatched += int((g != cams).any(axis=1).sum())
-        cams = g.copy()                          # keep both sides on the same state for the next step
+        diff = np.nonzero((g != cams).any(axis=1))[0]
+        mismatched += len(diff)
+        for o in diff:                           # a mismatching agent is off by one unit in the last place, in x or z only
+            d = np.abs(g[o, :5].astype(np.int64) - cams[o, :5].astype(np.int64))
+            assert d[1] == 0 and d[3] == 0 and d[4] == 0 and d[0] <= 1 and d[2] <= 1, (step, o, d)
+        cams = g.copy()                          # a 1-ulp difference could flip a later collision: continue from the GPU's state
         for o in range(cfg.num_obs):             # and the boxes the GPU now holds for those agents
             e = o // cfg.agents
             f = cams[o, :5].view(np.float32)
@@ -96,6 +100,7 @@ def test_move_agents_matches_oracle_then_renders(oracle):
             boxes[e, cams[o, 5], 3:6] = (f[:3] + np.float32([0.25, 0.25, 0.25])).view(np.int32)
     assert blocked > 10
     # double sin/cos differ by an ulp between libm and CUDA at most in rare roundings
+    print(f"move_agents: {mismatched} of {12 * cfg.num_obs} agent-steps differ from the oracle (each by <= 1 ulp)")
     assert mismatched <= 1, mismatched
     rgb, depth = batch.alloc_outputs()
     batch.render_batch(rgb, depth)               # no mv_set_cameras: the move rebuilt the ray bases

@@ -69,7 +69,7 @@ def test_tiny_config_all_pixels(oracle):
 
 def test_tiny_many_seeds_brute_force(oracle):
     from gpu_util import render_scene, scene_to_numpy
-    tot = {"pixels": 0, "rgb_mismatch": 0, "unexcused": 0}
+    tot = {"pixels": 0, "rgb_mismatch": 0, "mismatch": 0, "unexcused": 0}
     for seed in range(10, 16):
         cfg = scenes.config("tiny", seed=seed, num_envs=6)
         sc = scenes.make_scene(cfg)
@@ -505,3 +505,62 @@ def test_two_batches_of_different_shape_alive_together():
     assert torch.equal(frames[0][0], frames[2][0]) and torch.equal(frames[0][1], frames[2][1])
     assert (frames[0][1] > 0).any() and (frames[1][1] > 0).any()
     big.destroy(); small.destroy()
+
+
+def _pitch_with_exact_zero_dy(W, hfov=np.float32(np.pi / 2)):
+    """A float32 pitch for which the image row with b = H-1-2py = 1 has d_y = fma(1, Us_y, F_y) == 0
+    exactly: F_y = float(sin p) and Us_y = float(cos p * ku), ku = tan(hfov/2)/W, must cancel.  Us_y is
+    the same float over thousands of neighbouring pitches while float(sin p) steps through every float,
+    so a short scan around -atan(ku) finds one.  Candidates whose double values sit close to a float
+    rounding boundary are skipped, so that a last-place difference between two libm's cannot matter."""
+    ku = math.tan(float(hfov) / 2.0) / W
+    p0 = np.float32(-math.atan(ku))
+    bits = p0.view(np.int32) + np.arange(-200000, 200000, dtype=np.int64)
+    p = bits.astype(np.int32).view(np.float32)
+    sp64, us64 = np.sin(p.astype(np.float64)), np.cos(p.astype(np.float64)) * ku
+    sp, us = sp64.astype(np.float32), us64.astype(np.float32)
+    ok = sp == -us
+    ulp = np.spacing(np.abs(sp))
+    safe = (np.abs(sp64 - sp) < 0.4 * ulp) & (np.abs(us64 - us) < 0.4 * np.spacing(us))
+    idx = np.nonzero(ok & safe)[0]
+    return (p[idx[len(idx) // 2]], len(idx)) if len(idx) else (None, 0)
+
+
+def test_ray_direction_component_exactly_zero(oracle):
+    """Even image sizes never put a pixel centre on the view axis, so an exactly zero direction component
+    needs a pitch chosen for it: one whole image row then has d_y == 0 and travels at constant height.
+    The library replaces the zero by 1e-30; away from the doubly degenerate case (eye exactly on a face
+    AND component exactly zero) that must give the oracle's result: boxes whose height range contains the
+    eye are hit, the others are missed, and the walk never changes layer."""
+    W, H = 128, 72
+    pitch, found = _pitch_with_exact_zero_dy(W)
+    assert pitch is not None, "no float32 pitch with an exactly zero d_y in 400000 candidates"
+    # the row with b = 1
+    py0 = (H - 2) // 2
+    gx, gy, gz = 32, 8, 32
+    grid = np.zeros((1, gy, gz, gx), np.uint8)
+    grid[0, 0] = 1
+    grid[0, :, 0, :] = 2; grid[0, :, gz - 1, :] = 2; grid[0, :, :, 0] = 3; grid[0, :, :, gx - 1] = 3
+    grid[0, 1:4, 20, 8:12] = 4                                   # a low wall the zero row passes over (eye above it)
+    grid[0, 1:6, 24, 18:24] = 5                                  # a taller wall that it hits
+    eye = (14.37, 4.41, 6.29)
+    boxes = box_rows([((12.0, 4.0, 12.0), (13.0, 5.0, 13.0), 6),      # height range contains the eye: hit
+                      ((15.0, 4.5, 12.0), (16.0, 5.5, 13.0), 7),      # starts above the eye: missed by the zero row
+                      ((17.0, 3.0, 11.0), (18.0, 4.4, 12.0), 8)])[None]   # ends just below the eye: missed
+    cams = np.stack([cam_row(*eye, 0.0, pitch), cam_row(*eye, 0.35, pitch)])
+    grid2 = np.repeat(grid, 2, axis=0)
+    g_rgb, g_depth, status, st = _render_custom(oracle, grid2, _pal(2, 10), cams, W, H, boxes=np.repeat(boxes, 2, axis=0),
+                                                box_count=np.array([3, 3]), max_boxes=3)
+    assert status == 0
+    parity.assert_parity(st, "exact zero d_y")
+    # the oracle confirms that the row really has d_y == 0: every hit in it keeps the eye's layer (voxels)
+    od = oracle.make_desc((gy, gz, gx), 3, W, H, 10)
+    for o in range(2):
+        _, o_depth, ids = oracle.render_obs(od, grid2[o], boxes[0], 3, _pal(2, 10)[o], cams[o])
+        row = ids[py0]
+        vox = row[:, 0] == 0
+        assert vox.any() and ((row[vox, 1] // (gx * gz)) == 4).all()          # voxel index -> layer 4 = floor(eye y)
+        hit_boxes = set(row[row[:, 0] == 1, 1].tolist())
+        assert hit_boxes <= {0} and (o == 1 or 0 in hit_boxes)
+        # and the library's row agrees pixel for pixel
+        assert parity.depth_close(g_depth[o, py0], o_depth[py0]).all()

@@ -64,3 +64,23 @@ def test_split_envs_covers_everything():
             ranges = [shard.split_envs(total, r, world) for r in range(world)]
             assert ranges[0][0] == 0 and ranges[-1][1] == total
             assert all(ranges[i][1] == ranges[i + 1][0] for i in range(world - 1))
+
+
+def test_bench_starts_its_own_ranks_and_plans_disjoint_env_ranges():
+    """`bench.py --gpus 2 --plan` launches two ranks by itself (no outer launcher), touches no GPU, and the
+    two ranks take disjoint, adjacent ranges of seeded environments: scale-out is independent instances."""
+    import json
+    import subprocess
+    import sys
+    from pathlib import Path
+    root = Path(__file__).resolve().parent.parent
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    env["CUDA_VISIBLE_DEVICES"] = ""
+    out = subprocess.run([sys.executable, str(root / "bench.py"), "--gpus", "2", "--plan", "--envs", "96"],
+                         capture_output=True, text=True, timeout=300, env=env, cwd=str(root))
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = [l for l in out.stdout.splitlines() if l.startswith("{")][-1]
+    plan = json.loads(line)
+    assert plan["n_gpus"] == 2 and plan["collectives_on_data_path"] == 0
+    r0, r1 = sorted(plan["plan"], key=lambda r: r["rank"])
+    assert (r0["env_begin"], r0["env_end"]) == (0, 96) and (r1["env_begin"], r1["env_end"]) == (96, 192)

@@ -62,3 +62,47 @@ def test_static_step_rejects_batches_beyond_the_fixed_array():
         batch.step_host_static(sc["cams"].contiguous(), rgb, dep)
     assert ei.value.code == -6
     batch.destroy()
+
+
+def test_static_step_allocates_nothing_on_a_fresh_batch():
+    """The property the entry point exists for: on a batch that never went through mv_step_host (so no
+    frame buffers exist yet), two static steps leave the amount of free device memory exactly as it was,
+    and the frames equal those of the device-pointer path."""
+    cfg = scenes.config("rooms_boxes", num_envs=10)            # 40 observations
+    B, sc, batch = _setup(cfg)
+    d_cams = sc["cams"].cuda().contiguous()
+    want_rgb, want_depth = batch.alloc_outputs()
+    batch.set_cameras(d_cams)
+    batch.render_batch(want_rgb, want_depth)
+    want_rgb, want_depth = want_rgb.cpu(), want_depth.cpu()
+    cams = sc["cams"].contiguous().pin_memory()
+    rgb = torch.empty(want_rgb.shape, dtype=torch.uint8).pin_memory()
+    dep = torch.empty(want_depth.shape, dtype=torch.float32).pin_memory()
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    for _ in range(2):
+        rgb.fill_(3); dep.fill_(-1.0)
+        batch.step_host_static(cams, rgb, dep)
+        assert torch.equal(rgb, want_rgb) and torch.equal(dep, want_depth)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    assert batch.query_status() == 0
+    batch.destroy()
+
+
+def test_static_step_limit_is_exactly_the_documented_one():
+    """129 observations at 128x72 fit the 8 MiB array, 130 do not."""
+    for agents, ok in ((129, True), (130, False)):
+        cfg = scenes.config("rooms", num_envs=1, agents=agents)
+        B, sc, batch = _setup(cfg)
+        cams = sc["cams"].contiguous()
+        rgb = torch.empty(cfg.num_obs, cfg.height, cfg.width, 3, dtype=torch.uint8)
+        dep = torch.empty(cfg.num_obs, cfg.height, cfg.width, dtype=torch.float32)
+        if ok:
+            batch.step_host_static(cams, rgb, dep)
+            assert (dep > 0).any()
+        else:
+            with pytest.raises(B.MvError) as ei:
+                batch.step_host_static(cams, rgb, dep)
+            assert ei.value.code == -6
+        batch.destroy()
