@@ -185,6 +185,24 @@ def time_extras(batch, cfg, cams, rgb, depth, dev):
     batch.debug_occupancy_in_global(True)
     out["render_occupancy_in_global_ms"] = med(lambda: batch.render_batch(rgb, depth))
     batch.debug_occupancy_in_global(False)
+    # the vectorised step() wrapper at this size: move + collide, auto-reset of the ~1 % of environments whose
+    # 100-step episode ends (new worlds generated and uploaded), time-left bar, render; wall clock over 20 steps
+    env = vecenv.VecRenderEnv(cfg, 100, device=dev.index, phase=torch.arange(E) % 100)
+    env.reset()
+    for _ in range(2):
+        env.step(moves)
+    torch.cuda.synchronize(dev)
+    t0 = time.perf_counter()
+    n_steps, n_reset = 20, 0
+    for _ in range(n_steps):
+        _, _, done = env.step(moves)
+        n_reset += int(done.sum())
+    torch.cuda.synchronize(dev)
+    dt = time.perf_counter() - t0
+    out["vecenv_steps_per_s"] = n_steps / dt
+    out["vecenv_obs_per_s"] = n_steps * cfg.num_obs / dt
+    out["vecenv_envs_reset_per_step"] = n_reset / n_steps
+    env.close()
     return out
 
 

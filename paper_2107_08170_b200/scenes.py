@@ -227,11 +227,16 @@ def _world_rooms(rng: Rng, env, gx, gy, gz, P, n_lines=6, pitch=9, n_pillars=24)
     return height, M2, floor
 
 
-def make_worlds(cfg: SceneConfig, env_begin: int = 0, env_count: int | None = None, device="cpu"):
-    """Grid, palette and the per-column stack height for envs [env_begin, env_begin+env_count)."""
-    env_count = cfg.num_envs - env_begin if env_count is None else env_count
+def make_worlds(cfg: SceneConfig, env_begin: int = 0, env_count: int | None = None, device="cpu", env_ids=None):
+    """Grid, palette and the per-column stack height for envs [env_begin, env_begin+env_count), or for
+    the seeded environment ids listed in `env_ids` (any order, any values)."""
     rng = Rng(cfg.seed, device)
-    env = torch.arange(env_begin, env_begin + env_count, device=rng.device)
+    if env_ids is not None:
+        env = torch.as_tensor(env_ids, dtype=torch.int64).to(rng.device)
+        env_count = env.numel()
+    else:
+        env_count = cfg.num_envs - env_begin if env_count is None else env_count
+        env = torch.arange(env_begin, env_begin + env_count, device=rng.device)
     gx, gy, gz = cfg.grid
     P = cfg.palette_size
     if cfg.world == "rooms":
@@ -363,8 +368,8 @@ def walk_cameras(cfg: SceneConfig, worlds: dict, cams: torch.Tensor, step: int):
     return out
 
 
-def make_scene(cfg: SceneConfig, env_begin: int = 0, env_count: int | None = None, device="cpu"):
-    w = make_worlds(cfg, env_begin, env_count, device)
+def make_scene(cfg: SceneConfig, env_begin: int = 0, env_count: int | None = None, device="cpu", env_ids=None):
+    w = make_worlds(cfg, env_begin, env_count, device, env_ids)
     bc = make_boxes_and_cameras(cfg, w)
     return {**w, **bc}
 

@@ -5,89 +5,116 @@ environments are reset automatically, so the last frame of an episode is never r
 Scenario logic, rewards and object physics are outside this library: an "episode" here is a
 fixed number of steps, after which the environment gets a freshly generated world.  The
 time-left bar of Appendix A.2 is drawn through the GUI overlay.  Observations are zero-copy CUDA
-tensors owned by this object (Section 3.2: frames exposed directly as GPU-side tensors)."""
+tensors owned by this object (Section 3.2: frames exposed directly as GPU-side tensors).
+
+Built for thousands of environments: episode clocks, the time-left rectangles and the agent state
+live on the GPU; per step the host only learns which environments finished (one small read), then
+generates all of their new worlds in one batch and uploads them run by run of neighbouring
+environment indices."""
 from __future__ import annotations
 
-import numpy as np
 import torch
 
 from . import binding, scenes
 
 BAR_RGB = (250, 240, 30)
 BAR_ROWS = 2
+_GEN_CHUNK = 512            # environments generated per scene-generator call
 
 
 def time_bar_rects(steps_left, episode_len, width, agents):
     """int32 [E*agents][1][4] overlay records: a bar of BAR_ROWS rows whose length is the share of
-    the episode that is left, rounded down to whole pixels."""
+    the episode that is left, rounded down to whole pixels.  Runs on the device of its inputs."""
     steps_left = torch.as_tensor(steps_left, dtype=torch.int64)
-    episode_len = torch.as_tensor(episode_len, dtype=torch.int64)
+    episode_len = torch.as_tensor(episode_len, dtype=torch.int64).to(steps_left.device)
     x1 = (width * steps_left) // episode_len.clamp(min=1)
     x1 = x1.clamp(0, width).repeat_interleave(agents)
     n = x1.numel()
-    rec = torch.zeros(n, 1, 4, dtype=torch.int32)
-    rec[:, 0, 0] = 0                                   # x0 = 0, y0 = 0
-    rec[:, 0, 1] = x1.to(torch.int32) | (BAR_ROWS << 16)   # x1 (low half), y1 (high half)
+    rec = torch.zeros(n, 1, 4, dtype=torch.int32, device=steps_left.device)
+    rec[:, 0, 1] = x1.to(torch.int32) | (BAR_ROWS << 16)   # x1 (low half), y1 (high half); x0 = y0 = 0
     rec[:, 0, 2] = BAR_RGB[0] | (BAR_RGB[1] << 8) | (BAR_RGB[2] << 16)
     return rec
 
 
+def _runs(sorted_idx):
+    """[(start position, length)] of the runs of consecutive integers in a sorted list."""
+    out, i, n = [], 0, len(sorted_idx)
+    while i < n:
+        j = i
+        while j + 1 < n and sorted_idx[j + 1] == sorted_idx[j] + 1:
+            j += 1
+        out.append((i, j - i + 1))
+        i = j + 1
+    return out
+
+
 class VecRenderEnv:
-    def __init__(self, cfg: scenes.SceneConfig, episode_len, device: int = 0, time_bar: bool = True):
+    def __init__(self, cfg: scenes.SceneConfig, episode_len, device: int = 0, time_bar: bool = True, phase=None):
+        """episode_len: steps per episode (scalar or one per env).  phase: optional initial value of each
+        env's step clock (so that episodes end at different times from the start)."""
         self.cfg, self.device = cfg, torch.device("cuda", device)
         E = cfg.num_envs
-        self.episode_len = torch.as_tensor(episode_len, dtype=torch.int64).expand(E).clone()
+        self.episode_len = torch.as_tensor(episode_len, dtype=torch.int64).expand(E).clone().to(self.device)
         self.time_bar = time_bar
         self.batch = binding.Batch(binding.desc_from_config(cfg, device, max_overlay_rects=1 if time_bar else 0))
         self.cams = torch.zeros(cfg.num_obs, 6, dtype=torch.int32, device=self.device)
         self.rgb, self.depth = self.batch.alloc_outputs()
-        self.t = torch.zeros(E, dtype=torch.int64)
-        self.episode = torch.zeros(E, dtype=torch.int64)
+        self.t = torch.zeros(E, dtype=torch.int64, device=self.device)
+        if phase is not None:
+            self.t = torch.as_tensor(phase, dtype=torch.int64).expand(E).clone().to(self.device)
+        self.episode = torch.zeros(E, dtype=torch.int64, device=self.device)
+        self._bar_count = torch.ones(cfg.num_obs, dtype=torch.int32, device=self.device)
         self._started = False
 
-    # env e in its k-th episode uses the seeded scene id e + k * num_envs
-    def _load_env(self, e: int):
+    def _load_envs(self, envs):
+        """Fresh worlds for the (sorted) local env indices in `envs`; env e in its k-th episode uses the
+        seeded scene id e + k * num_envs."""
         cfg, A = self.cfg, self.cfg.agents
-        sc = scenes.make_scene(cfg, e + int(self.episode[e]) * cfg.num_envs, 1, device=self.device)
-        boxes = count = None
-        if cfg.max_boxes > 0:
-            boxes, count = sc["boxes"].contiguous(), sc["box_count"].contiguous()
-        self.batch.upload_worlds(e, 1, sc["grid"].contiguous(), boxes, count, sc["palette"].contiguous())
-        self.cams[e * A:(e + 1) * A] = sc["cams"]
+        envs = [int(e) for e in envs]
+        ep = self.episode.cpu()
+        for c0 in range(0, len(envs), _GEN_CHUNK):
+            chunk = envs[c0:c0 + _GEN_CHUNK]
+            ids = torch.tensor([e + int(ep[e]) * cfg.num_envs for e in chunk], dtype=torch.int64)
+            sc = scenes.make_scene(cfg, device=self.device, env_ids=ids)
+            for i0, n in _runs(chunk):
+                boxes = count = None
+                if cfg.max_boxes > 0:
+                    boxes, count = sc["boxes"][i0:i0 + n].contiguous(), sc["box_count"][i0:i0 + n].contiguous()
+                self.batch.upload_worlds(chunk[i0], n, sc["grid"][i0:i0 + n].contiguous(), boxes, count,
+                                         sc["palette"][i0:i0 + n].contiguous())
+            obs = (torch.tensor(chunk, device=self.device)[:, None] * A + torch.arange(A, device=self.device)).flatten()
+            self.cams[obs] = sc["cams"]
 
     def _render(self):
         if self.time_bar:
             rects = time_bar_rects(self.episode_len - self.t, self.episode_len, self.cfg.width, self.cfg.agents)
-            count = torch.ones(self.cfg.num_obs, dtype=torch.int32)
-            self.batch.set_overlays(rects.to(self.device), count.to(self.device))
+            self.batch.set_overlays(rects, self._bar_count)
         self.batch.render_batch(self.rgb, self.depth)
         return self.rgb, self.depth
 
     def reset(self):
         """Only needed once, right after construction."""
-        for e in range(self.cfg.num_envs):
-            self._load_env(e)
-        self.t.zero_()
+        self._load_envs(range(self.cfg.num_envs))
         self.batch.set_cameras(self.cams)
         self._started = True
         return self._render()
 
     def step(self, moves: torch.Tensor):
         """moves: CUDA float32 [num_obs][4] = (forward, strafe, dyaw, dpitch).  Returns
-        (rgb [O][H][W][3] uint8, depth [O][H][W] float32, done [E] bool); for a finished env the
-        frames already show the first view of its next episode."""
+        (rgb [O][H][W][3] uint8, depth [O][H][W] float32, done [E] bool on the GPU); for a finished env
+        the frames already show the first view of its next episode."""
         assert self._started, "call reset() once before step()"
         self.batch.move_agents(self.cams, moves.contiguous())
         self.t += 1
         done = self.t >= self.episode_len
-        if bool(done.any()):
-            for e in torch.nonzero(done).flatten().tolist():
-                self.episode[e] += 1
-                self.t[e] = 0
-                self._load_env(e)
+        finished = torch.nonzero(done).flatten().cpu().tolist()       # the one device->host read of a step
+        if finished:
+            self.episode[done] += 1
+            self.t[done] = 0
+            self._load_envs(finished)
             self.batch.set_cameras(self.cams)
         rgb, depth = self._render()
-        return rgb, depth, done.clone()
+        return rgb, depth, done
 
     def close(self):
         self.batch.destroy()
