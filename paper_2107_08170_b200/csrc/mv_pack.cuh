@@ -43,13 +43,14 @@ __global__ void pack_grid_kernel(const uint8_t *__restrict__ grid, unsigned char
     const size_t env = (size_t)env_begin + e;
     const uint32_t u0 = voxel_index(lay.ysh, gx, 4 * xg, 32 * wq, z);
     uint8_t *mdst = mat + env * ((size_t)gx * gz << lay.ysh) + u0;
+    uint32_t col[4][8];                                 // material bytes: column c, heights 4k..4k+3 in word k
 #pragma unroll
     for (int h0 = 0; h0 < 32; h0 += 4) {
         uint32_t v[4], t[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int y = 32 * wq + h0 + i;
-            const uint32_t orig = y < gy ? *reinterpret_cast<const uint32_t *>(src + (size_t)y * gz * gx) : 0u;
+            const uint32_t orig = y < gy ? __ldg(reinterpret_cast<const uint32_t *>(src + (size_t)y * gz * gx)) : 0u;
             const uint32_t nz = __vcmpne4(orig, 0u);               // 0xff per filled byte, decided before clamping
 #pragma unroll
             for (int c = 0; c < 4; ++c) bits[c] |= ((nz >> (8 * c)) & 1u) << (h0 + i);
@@ -59,8 +60,13 @@ __global__ void pack_grid_kernel(const uint8_t *__restrict__ grid, unsigned char
         }
         transpose4x4(v, t);
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-            *reinterpret_cast<uint32_t *>(mdst + ((size_t)c << lay.ysh) + h0) = t[c];
+        for (int c = 0; c < 4; ++c) col[c][h0 / 4] = t[c];
+    }
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {                       // 32 contiguous bytes per column: two 16-byte stores
+        uint4 *dst = reinterpret_cast<uint4 *>(mdst + ((size_t)c << lay.ysh));
+        dst[0] = make_uint4(col[c][0], col[c][1], col[c][2], col[c][3]);
+        dst[1] = make_uint4(col[c][4], col[c][5], col[c][6], col[c][7]);
     }
     uint32_t *occ = reinterpret_cast<uint32_t *>(env_blocks + env * lay.stride);
 #pragma unroll
