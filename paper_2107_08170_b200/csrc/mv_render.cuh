@@ -422,10 +422,12 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     keep(lane_a); keep(lane_b); keep(st_src); keep(st_sel);
     const uint32_t tile_begin = smem_addr(s_tile) + 16u * (uint32_t)warp;
 #if MV_PROBE == 3
-    const uint32_t tile_end = smem_addr(s_tile);
+    uint32_t tile_end = smem_addr(s_tile);
 #else
-    const uint32_t tile_end = smem_addr(s_tile) + 16u * (uint32_t)ntiles;
+    uint32_t tile_end = smem_addr(s_tile) + 16u * (uint32_t)ntiles;
 #endif
+    uint32_t mask_step = 4u * kWarps * (uint32_t)mw;                        // bytes between a warp's consecutive tile masks
+    keep(tile_end); keep(mask_step);
 
     for (int ag = 0; ag < apc; ++ag) {
         const int obs = obs0 + ag;
@@ -440,6 +442,8 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         const float Px = c0.x, Py = c0.y, Pz = c0.z;
         const bool cam_in = (aflags & kAgentInside) != 0;
         const int ov_count = __float_as_int(c3.w);
+        uint32_t rare = (mw > 1 ? 1u : 0u) | (ov_count > 0 ? 2u : 0u);     // non-zero: every tile takes the slow branch
+        keep(rare);
         uint32_t abase = smem_addr(agent_rec(ag));
         uint32_t mask_p = smem_addr(agent_mask(ag) + (size_t)warp * mw);
         // (store addresses as global-space addresses for the PTX store block)
@@ -449,7 +453,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         asm volatile("" : "+l"(depth_lane), "+l"(rgb_lane));
 
         // ---- tiles: warp w takes tiles w, w + nwarps, ... (8 x 4 pixels, one per lane)
-        for (uint32_t tile_p = tile_begin; tile_p < tile_end; tile_p += 16u * kWarps, mask_p += 4u * kWarps * (uint32_t)mw) {
+        for (uint32_t tile_p = tile_begin; tile_p < tile_end; tile_p += 16u * kWarps, mask_p += mask_step) {
             int tile_px;
             uint32_t pos, bit = 0, row, sgn3;
             float t_hit, dtx, dty, dtz;
@@ -676,8 +680,9 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             m = 0;
 #endif
 
-            // ---- boxes of this tile; a box wins only with a strictly smaller time
-            {
+            // ---- the less common work, behind one test: boxes binned to this tile (or more than 32 boxes
+            // per environment) and the GUI overlay.  A box wins only with a strictly smaller time.
+            if ((m | rare) != 0u) {
                 if (m != 0u || mw > 1) {
                     // signed reciprocals again, and the ray's rows of the DDA table for the faces
                     const float ix = __uint_as_float(__float_as_uint(dtx) | (sgn3 << 31));
@@ -717,17 +722,16 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                         depth = tb + 0.0f;
                     }
                 }
-            }
-
-            // ---- GUI overlay: rectangles in list order, later ones on top; depth is left alone
-            if (ov_count > 0) {
-                const uint32_t tile_no = (tile_p - smem_addr(s_tile)) >> 4;
-                if ((agent_ovtile(ag)[tile_no >> 5] >> (tile_no & 31)) & 1u) {
-                    const int4 *ov = agent_ov(ag);
-                    const int px = (tile_px % W) + (lane & 7), py = (tile_px / W) + (lane >> 3);
-                    for (int r = 0; r < ov_count; ++r) {
-                        const int4 q = ov[2 * r];
-                        if (px >= q.x && px < q.z && py >= q.y && py < q.w) rgbx = (uint32_t)ov[2 * r + 1].x;
+                // GUI overlay: rectangles in list order, later ones on top; depth is left alone
+                if (ov_count > 0) {
+                    const uint32_t tile_no = (tile_p - smem_addr(s_tile)) >> 4;
+                    if ((agent_ovtile(ag)[tile_no >> 5] >> (tile_no & 31)) & 1u) {
+                        const int4 *ov = agent_ov(ag);
+                        const int px = (tile_px % W) + (lane & 7), py = (tile_px / W) + (lane >> 3);
+                        for (int r = 0; r < ov_count; ++r) {
+                            const int4 q = ov[2 * r];
+                            if (px >= q.x && px < q.z && py >= q.y && py < q.w) rgbx = (uint32_t)ov[2 * r + 1].x;
+                        }
                     }
                 }
             }
