@@ -109,10 +109,13 @@ typedef struct mv_batch_desc {
     int32_t num_envs;                   /* N >= 1 */
     int32_t agents_per_env;             /* M >= 1 */
     int32_t grid_x, grid_y, grid_z;     /* voxels per axis; each a multiple of 4, 4..1024.
-                                           Up to about 1.6 M voxels per env the occupancy bits
-                                           (grid_x*grid_y*grid_z/8 bytes) are staged in shared
-                                           memory; larger grids are read from global memory
-                                           (slower per step, same results) */
+                                           The occupancy bits are kept packed along y, one
+                                           column of h bits per (x, z), h = the power of two
+                                           >= grid_y, at least 32.  While grid_x*grid_z*h/8 bytes
+                                           plus the per-env tables fit in shared memory (about
+                                           200 KB) they are staged there; larger grids are read
+                                           from global memory (slower per step, same results).
+                                           Grids up to 32 high take the fastest traversal. */
     int32_t max_boxes;                  /* per env, agent bodies included; 0..256 */
     int32_t width, height;              /* pixels; width a multiple of 8, height of 4; <= 4096 */
     int32_t palette_size;               /* 1..256 entries per env */
@@ -170,7 +173,8 @@ int mv_render_batch(mv_batch *batch, uint8_t *d_rgb, float *d_depth, void *cuda_
  *   d_boxes_out DEVICE mv_box [env_count][max_out]; box b of an env is valid for b < min(count, max_out)
  *   d_count_out DEVICE int32 [env_count]; the number of boxes the sweep produces (may exceed max_out,
  *               in which case only the first max_out were written)
- * The first call allocates a scratch bitmap (1 bit per voxel for as many envs as fit in 256 MiB).
+ * The first call allocates scratch (2 bits per voxel for as many envs as fit in 256 MiB: the
+ * coverage bitmap and a copy of the occupancy in sweep order).
  * Errors: INVALID_ARG, NOT_READY (an env in the range has no grid), OUT_OF_MEMORY, CUDA. */
 int mv_merge_voxels(mv_batch *batch, int env_begin, int env_count, mv_box *d_boxes_out,
                     int32_t *d_count_out, int max_out, void *cuda_stream);
@@ -211,8 +215,10 @@ int mv_move_agents(mv_batch *batch, mv_camera *d_cams_inout, const mv_agent_move
  *   h_box_count HOST int32 [num_envs]; required when h_boxes is given
  *   h_rgb, h_depth HOST outputs, same shapes as mv_render_batch; page-locked memory is
  *               needed for the copies to overlap
- * The first call allocates device-side frame buffers of the batch's full output size.
- * Errors: as the calls it is made of. */
+ * The first call allocates device-side frame buffers of the batch's full output size (all of
+ * them or, on failure, none: a failed first call can be retried).
+ * Errors: as the calls it is made of; DEVICE_TIMEOUT if a bounded device-side wait ran out during
+ * the step (the frames are then not valid; the flag stays set until mv_query_status clears it). */
 int mv_step_host(mv_batch *batch, const mv_camera *h_cams, const mv_box *h_boxes,
                  const int32_t *h_box_count, uint8_t *h_rgb, float *h_depth, void *cuda_stream);
 
@@ -234,12 +240,13 @@ int mv_step_host(mv_batch *batch, const mv_camera *h_cams, const mv_box *h_boxes
  * The first call on each device looks up the array's device address (a runtime query, not an
  * allocation); make that first call before starting any stream capture.
  * The array is shared by every batch and every call on that device and keeps whatever the last
- * call left in it.  Nothing in it needs clearing, because each call overwrites every byte it
- * later reads; but two calls whose device work overlaps (different streams, or different
+ * call left in it.  Nothing in it needs clearing, because each call that returns MV_OK has
+ * overwritten every byte it read back; but two calls whose device work overlaps (different streams, or different
  * threads) race on it, so serialise them.  Synchronous like mv_step_host.
  * Calls no cudaMalloc, cudaFree or other allocating routine.
  * Errors: INVALID_ARG, NOT_READY, UNSUPPORTED (batch too large for the array, device ordinal
- * >= 64), CUDA. */
+ * >= 64), DEVICE_TIMEOUT (as mv_step_host; the array may then hold an earlier call's frames),
+ * CUDA. */
 int mv_step_host_static(mv_batch *batch, const mv_camera *h_cams, uint8_t *h_rgb, float *h_depth,
                         void *cuda_stream);
 
