@@ -161,6 +161,7 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
 #define MV_MINB 3
 #endif
 
+constexpr uint32_t kOverlayTileBit = 0x80000000u;   // in a tile's box mask word (only when max_boxes < 32)
 constexpr uint32_t kAgentInside = 1u;      // eye inside the occupied cell box
 constexpr uint32_t kAgentBad = 2u;         // non-finite camera: sky frame
 constexpr uint32_t kAgentFilled = 4u;      // the eye's own voxel is filled
@@ -273,6 +274,9 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                     for (int tx = cx0 >> 3; tx <= ((cx1 - 1) >> 3); ++tx) {
                         const int t = ty * p.tiles_x + tx;
                         atomicOr(&agent_ovtile(ag)[t >> 5], 1u << (t & 31));
+                        // with fewer than 32 boxes the top bit of the tile's box mask is free: it sends
+                        // exactly the touched tiles down the slow branch
+                        if (p.max_boxes < 32) atomicOr(&agent_mask(ag)[t], kOverlayTileBit);
                     }
         }
     }
@@ -442,7 +446,9 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         const float Px = c0.x, Py = c0.y, Pz = c0.z;
         const bool cam_in = (aflags & kAgentInside) != 0;
         const int ov_count = __float_as_int(c3.w);
-        uint32_t rare = (mw > 1 ? 1u : 0u) | (ov_count > 0 ? 2u : 0u);     // non-zero: every tile takes the slow branch
+        // non-zero: every tile takes the slow branch (more than one mask word per tile, or an overlay that
+        // cannot flag its tiles in the box mask)
+        uint32_t rare = (mw > 1 ? 1u : 0u) | ((ov_count > 0 && p.max_boxes >= 32) ? 2u : 0u);
         keep(rare);
         uint32_t abase = smem_addr(agent_rec(ag));
         uint32_t mask_p = smem_addr(agent_mask(ag) + (size_t)warp * mw);
@@ -683,6 +689,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             // ---- the less common work, behind one test: boxes binned to this tile (or more than 32 boxes
             // per environment) and the GUI overlay.  A box wins only with a strictly smaller time.
             if ((m | rare) != 0u) {
+                if (p.max_boxes < 32) m &= ~kOverlayTileBit;
                 if (m != 0u || mw > 1) {
                     // signed reciprocals again, and the ray's rows of the DDA table for the faces
                     const float ix = __uint_as_float(__float_as_uint(dtx) | (sgn3 << 31));
