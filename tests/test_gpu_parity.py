@@ -564,3 +564,30 @@ def test_ray_direction_component_exactly_zero(oracle):
         assert hit_boxes <= {0} and (o == 1 or 0 in hit_boxes)
         # and the library's row agrees pixel for pixel
         assert parity.depth_close(g_depth[o, py0], o_depth[py0]).all()
+
+
+def test_host_step_allocation_failure_is_reported_and_can_be_retried():
+    """mv_step_host allocates its device-side frame buffers on first use.  When that cannot be satisfied
+    (here: 100,000 observations of 640x480, over 200 GB of frames) the call reports OUT_OF_MEMORY, keeps
+    nothing half-allocated, and a second call fails the same clean way instead of launching on null
+    pointers.  No kernel runs in this test."""
+    B = _binding()
+    E = 100000
+    desc = B.make_desc(E, 1, (4, 4, 4), 0, 640, 480, 2)
+    batch = B.Batch(desc)
+    dev = torch.device("cuda", 0)
+    batch.upload_worlds(0, E, torch.zeros(E, 4, 4, 4, dtype=torch.uint8, device=dev), None, None,
+                        torch.zeros(E, 2, 3, dtype=torch.uint8, device=dev))
+    cams = torch.zeros(E, 6, dtype=torch.int32)
+    rgb = torch.zeros(16, dtype=torch.uint8)          # never touched: the allocation fails before any copy
+    depth = torch.zeros(16, dtype=torch.float32)
+    for _ in range(2):
+        with pytest.raises(B.MvError) as ei:
+            batch.step_host(cams, rgb, depth)
+        assert ei.value.code == -2
+    assert batch.query_status() == 0
+    batch.destroy()
+    # the context is intact: an ordinary batch still renders
+    from gpu_util import render_scene
+    cfg = scenes.config("tiny")
+    assert render_scene(cfg, scenes.make_scene(cfg))[2] == 0
