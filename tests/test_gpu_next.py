@@ -183,3 +183,56 @@ def test_merged_boxes_render_like_the_grid_on_gpu(oracle):
     same = (rgb_g == rgb_b).all(dim=-1) & ((depth_g - depth_b).abs() <= 1e-4 * depth_g.clamp(min=1e-3))
     assert float(same.float().mean()) > 0.999
     batch.destroy(); bb.destroy()
+
+
+def test_tall_grid_with_multi_word_columns(oracle):
+    """Grids more than 32 voxels high keep several occupancy words per (x, z) column and take the indexed
+    flavour of the walk; render, merge and agent motion all address voxels through the same index."""
+    from paper_2107_08170_b200 import binding as B
+    from gpu_util import upload_scene, scene_to_numpy
+    from helpers import cam_row
+    cfg = scenes.config("tiny", grid=(16, 40, 20), num_envs=3, seed=7, movable_boxes=3)
+    sc = scenes.make_scene(cfg)
+    rng = np.random.default_rng(5)
+    grid = sc["grid"].numpy().copy()
+    grid[:, 30:38, 3:9, 5:9] = rng.integers(0, 4, size=(3, 8, 6, 4)).astype(np.uint8)   # voxels above height 32
+    sc["grid"] = torch.from_numpy(grid)
+    cams = sc["cams"].numpy().copy()
+    cams[1, :5] = np.array([8.3, 34.2, 12.7, 2.6, -0.4], np.float32).view(np.int32)      # an eye up there, looking down
+    cams[2, :5] = np.array([-3.0, 45.0, 9.5, 1.2, -0.7], np.float32).view(np.int32)      # and one outside the grid
+    sc["cams"] = torch.from_numpy(cams)
+    batch = B.Batch(B.desc_from_config(cfg))
+    upload_scene(batch, sc)
+    batch.set_cameras(sc["cams"].cuda())
+    rgb, depth = batch.alloc_outputs()
+    batch.render_batch(rgb, depth)
+    assert batch.query_status() == 0
+    st = parity.compare_scene(oracle, cfg, scene_to_numpy(sc), range(cfg.num_obs), rgb.cpu().numpy(), depth.cpu().numpy())
+    parity.assert_parity(st, "tall grid")
+    assert (depth[1] > 0).float().mean() > 0.5
+    # the same frames with the occupancy read from global memory
+    rgb2, depth2 = batch.alloc_outputs()
+    batch.debug_occupancy_in_global(True)
+    batch.render_batch(rgb2, depth2)
+    batch.debug_occupancy_in_global(False)
+    assert torch.equal(rgb, rgb2) and torch.equal(depth, depth2)
+    # merge: same boxes, same order as the serial sweep
+    boxes, counts = batch.merge_voxels(0, 3, 512)
+    for e in range(3):
+        want, total = oracle.merge_voxels(grid[e], cfg.palette_size, 512)
+        assert int(counts[e]) == total and (boxes[e, :len(want)].cpu().numpy() == want).all()
+    # agent motion: collision against voxels above height 32
+    d_cams = torch.from_numpy(np.stack([cam_row(7.0, 33.0, 2.0, 0.0, 0.0), cam_row(7.0, 20.0, 2.0, 0.0, 0.0),
+                                        cam_row(7.0, 33.0, 2.0, 0.0, 0.0)])).cuda()
+    solid = np.zeros_like(grid); solid[:, 30:38, 3:9, 5:9] = 1
+    sc2 = dict(sc, grid=torch.from_numpy(np.where(solid > 0, 1, 0).astype(np.uint8)))
+    upload_scene(batch, sc2)
+    moves = torch.tensor([[2.0, 0, 0, 0]] * 3, dtype=torch.float32).cuda()
+    batch.move_agents(d_cams, moves)
+    after = d_cams.cpu().numpy()[:, :5].view(np.float32)
+    for o in range(3):
+        new, _ = oracle.move_agent(sc2["grid"][o].numpy(), np.array([7.0, 33.0 if o != 1 else 20.0, 2.0, 0.0, 0.0], np.float32),
+                                   np.array([2.0, 0, 0, 0], np.float32), (0.25, 0.75, 0.25), 1.0)
+        assert (after[o] == new).all(), (o, after[o], new)
+    assert after[0, 2] == 2.0 and after[1, 2] == 4.0          # blocked by the block at z = 3 up there, free below it
+    batch.destroy()
