@@ -8,10 +8,11 @@
 // masks and writes the tile table.  Each agent's boxes are then binned to 8x4-pixel screen tiles
 // by the bounding rectangle of their projected corners (conservative, so every box that a
 // pixel's ray can touch is tested for that pixel).  Tiles are dealt to warps round-robin; each
-// lane owns one pixel of the tile: it walks the occupancy grid with a branch-free 3D-DDA in
-// shared memory, tests the tile's candidate boxes with slab tests, looks the colour up in the
-// shaded table and the warp writes 24-byte RGB row segments as packed 32-bit words and 32-byte
-// depth row segments.
+// lane owns one pixel of the tile: it walks the occupancy grid (packed along y: a column of up to
+// 32 voxels is one word) with a predicated 3D-DDA in shared memory, tests the tile's candidate
+// boxes with slab tests, looks the colour up in the shaded table and the warp writes 24-byte RGB
+// row segments as packed 32-bit words and 32-byte depth row segments.  The common case runs in
+// three blocks of PTX (ray set-up + walk, colour, stores); everything rarer is C++ around them.
 // The walk is confined to the cell box that holds every filled voxel of the environment (built at
 // upload), so rays that leave it stop at once; GUI rectangles, if any, are painted over the colour
 // just before the store.
@@ -154,6 +155,9 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
     " .reg .b64 ag, gbase;\n"                        \
     " mov.f32 ns, 0f00000000;\n"
 
+// MV_PROBE builds are for instruction counting only (never the shipped library): 1 = every walk ends
+// at its first test, 2 = also no box tests, 3 = no tiles at all (CTA prologue alone), 9 = the depth
+// channel carries each ray's number of walk steps instead of depth.
 #ifndef MV_PROBE
 #define MV_PROBE 0
 #endif
