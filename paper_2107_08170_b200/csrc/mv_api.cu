@@ -112,7 +112,10 @@ mv_batch::Smem smem_layout(const mv_batch *b, int apc) {
     m.agent_ovtile_off = m.agent_mask_off + round_up(ntiles * (uint32_t)b->mask_words * 4, 16);
     m.agent_stride = m.agent_ovtile_off + round_up(((ntiles + 31) / 32) * 4, 16);
     m.misc_off = m.agent_off + (uint32_t)apc * m.agent_stride;
-    m.bytes = m.misc_off + 16;
+    m.bytes = m.misc_off + 32;
+#if defined(MV_BRICKS) && MV_BRICKS == 1
+    m.bytes += round_up((uint32_t)((d.grid_x / 4) * (d.grid_z / 4)), 16);   // experiment: one byte per column of 4x4x4 bricks
+#endif
     return m;
 }
 

@@ -161,6 +161,13 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
 #ifndef MV_PROBE
 #define MV_PROBE 0
 #endif
+// MV_BRICKS builds are an experiment, never the shipped library: 1 = two-level traversal (a one-bit map
+// of 4x4x4 bricks built per CTA; empty bricks are jumped across, occupied ones walked cell by cell by
+// the same PTX loop), 2 = the flat walk through the same C++ path, as the like-for-like baseline of 1.
+// Both need grid_x to be a power of two and a grid at most 32 high.
+#ifndef MV_BRICKS
+#define MV_BRICKS 0
+#endif
 #ifndef MV_MINB
 #define MV_MINB 3
 #endif
@@ -407,6 +414,21 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                     atomicOr(&mask[(ty * p.tiles_x + tx) * mw + (b >> 5)], bit);
         }
     }
+#if MV_BRICKS == 1
+    unsigned char *s_brick = smem + p.smem_misc_off + 32;
+    if (COLW) {
+        const int bxn = gx >> 2, bzn = gz >> 2;
+        for (int i = tid; i < bxn * bzn; i += NT) {
+            const int bx = i % bxn, bz = i / bxn;
+            uint32_t m = 0;
+            for (int j = 0; j < 4; ++j)
+                for (int k = 0; k < 4; ++k) m |= s_occ[(4 * bx + k) + gx * (4 * bz + j)];
+            uint32_t byte = 0;
+            for (int by = 0; by < 8; ++by) byte |= ((m >> (4 * by)) & 0xFu) ? (1u << by) : 0u;
+            s_brick[i] = (unsigned char)byte;
+        }
+    }
+#endif
     __syncthreads();
 
     const float flox = (float)lox, floy = (float)loy, floz = (float)loz;
@@ -467,7 +489,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             int tile_px;
             uint32_t pos, bit = 0, row, sgn3;
             float t_hit, dtx, dty, dtz;
-            if (COLW && cam_in) {
+            if (COLW && cam_in && !MV_BRICKS) {
                 // ---- the common case in one block of PTX: tile record, ray through the pixel centre
                 // (d = F + a*Rs + b*Us, a = 2px+1-W, b = H-1-2py, two chained FMAs per component; a
                 // component that is exactly zero becomes 1e-30 so that it never crosses a cell face and
@@ -635,6 +657,61 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
 #define MV_DDA_OUTS                                                                                       \
                     " selp.u32 a, 16, 32, py;\n selp.u32 a, 0, a, px;\n add.u32 a, a, %15;\n"                        \
                     " @ph ld.shared.u32 %3, [a+" MV_TAB_ROW "];\n mov.b32 %0, pos;\n mov.b32 %1, bit;\n mov.f32 %2, thit;\n"
+#if MV_BRICKS == 1
+                if (COLW && cam_in) {
+                    // two-level traversal: per brick, its exit time; occupied bricks are walked by the PTX
+                    // loop up to that time, then every axis is advanced past its crossings up to it (one
+                    // crossing after a walked brick, several across an empty one) and the arrival cell tested
+                    const int lgx = 31 - __clz(gx);
+                    const float adx = fabsf(dx), ady = fabsf(dy), adz = fabsf(dz);
+                    const float t_exit_all = t_exit;
+                    for (int guard = 0; guard < 3 * 256 + 8 && row == kNoRow; ++guard) {
+                        const uint32_t col = (pos - occ_base) >> 2;
+                        const int cx = (int)(col & (uint32_t)(gx - 1)), cz = (int)(col >> lgx), cy = 31 - __clz(bit);
+                        const int nbx = (sgn3 & 1u) ? (cx & 3) : 3 - (cx & 3), nby = (sgn3 & 2u) ? (cy & 3) : 3 - (cy & 3);
+                        const int nbz = (sgn3 & 4u) ? (cz & 3) : 3 - (cz & 3);
+                        const float tbk = min3f(fmaf((float)nbx, dtx, t0x), fmaf((float)nby, dty, t0y), fmaf((float)nbz, dtz, t0z));
+                        if ((s_brick[(cx >> 2) + (gx >> 2) * (cz >> 2)] >> (cy >> 2)) & 1u) {
+                            t_exit = fminf(tbk, t_exit_all);
+                            asm volatile("{\n" MV_DDA_DECL MV_DDA_IN MV_DDA_LOOP(MV_DDA_STEP_COLW) MV_DDA_OUTS
+                                         " mov.f32 %4, tx;\n mov.f32 %5, ty;\n mov.f32 %6, tz;\n}\n"
+                                         : "+r"(pos), "+r"(bit), "+f"(t_hit), "+r"(row), "+f"(t0x), "+f"(t0y), "+f"(t0z)
+                                         : "f"(dtx), "f"(dty), "f"(dtz), "r"(sx), "r"(sy), "r"(sz), "f"(t_exit), "r"(p.max_steps),
+                                           "r"(tab), "l"(s_occ)
+                                         : "memory");
+                            if (row != kNoRow) break;
+                        }
+                        if (tbk >= t_exit_all) break;
+                        // crossings of each axis up to the brick's exit time (with a tolerance: the exit
+                        // time is a product, the crossing times are sums)
+                        const float tol = fmaf(tbk, 1e-5f, 1e-6f);
+                        const int mx = t0x <= tbk + tol ? (int)floorf(fmaxf(tbk - t0x, 0.0f) * adx + 1e-3f) + 1 : 0;
+                        const int my = t0y <= tbk + tol ? (int)floorf(fmaxf(tbk - t0y, 0.0f) * ady + 1e-3f) + 1 : 0;
+                        const int mz = t0z <= tbk + tol ? (int)floorf(fmaxf(tbk - t0z, 0.0f) * adz + 1e-3f) + 1 : 0;
+                        // nothing to cross: the walk itself took the step out of the brick (its crossing times are
+                        // sums, the brick's exit time a product); look at the new brick
+                        if (mx + my + mz == 0) continue;
+                        // never past the occupied cell box (integer test, so the position stays valid)
+                        const int rx = (sgn3 & 1u) ? cx - lox : hix - 1 - cx, ry = (sgn3 & 2u) ? cy - loy : hiy - 1 - cy;
+                        const int rz = (sgn3 & 4u) ? cz - loz : hiz - 1 - cz;
+                        if (mx > rx || my > ry || mz > rz) break;
+                        t0x = fmaf((float)mx, dtx, t0x); t0y = fmaf((float)my, dty, t0y); t0z = fmaf((float)mz, dtz, t0z);
+                        pos += (uint32_t)(mx * sx + mz * sz);
+                        bit = __funnelshift_l(bit, bit, (uint32_t)(my * sy) & 31u);
+                        if (pos - occ_base >= p.lay.occ_bytes) break;        // (cannot happen; guards the load below)
+                        uint32_t w;
+                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(pos));
+                        if (w & bit) {
+                            t_hit = tbk;
+                            const float lastx = t0x - dtx, lasty = t0y - dty, lastz = t0z - dtz;     // the latest crossing taken
+                            const float lx_ = mx ? lastx : -kInf, ly_ = my ? lasty : -kInf, lz_ = mz ? lastz : -kInf;
+                            const float latest = fmaxf(lx_, fmaxf(ly_, lz_));
+                            asm volatile("ld.shared.u32 %0, [%1+" MV_TAB_ROW "];" : "=r"(row)
+                                         : "r"(tab + (lx_ == latest ? 0u : (ly_ == latest ? 16u : 32u))));
+                        }
+                    }
+                } else
+#endif
                 if constexpr (COLW) {
                     asm volatile("{\n" MV_DDA_DECL MV_DDA_IN MV_DDA_LOOP(MV_DDA_STEP_COLW) MV_DDA_OUTS "}\n" MV_DDA_IO);
                 } else if constexpr (OCC_SHARED) {
