@@ -133,7 +133,10 @@ def cpu_model() -> str:
     return "unknown"
 
 
-def cpu_oracle_rate(cfg, kept, max_seconds=25.0, max_obs=8):
+CPU_SAMPLE_OBS = 32      # observations the oracle renders for the cpu_baseline figure (about 10 s on 16 cores)
+
+
+def cpu_oracle_rate(cfg, kept, max_seconds=25.0, max_obs=CPU_SAMPLE_OBS):
     """Observations per second of the oracle, as it stands, on this host's cores."""
     from oracle import mv_oracle
     mv_oracle.build()
@@ -339,7 +342,7 @@ def main():
     # workloads whose per-step bytes do not dwarf the 126 MB L2 get an L2 flush between timed steps
     step_bytes = workload.algorithmic_bytes(cfg)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if step_bytes < (512 << 20) else None
-    keep = list(range(0, cfg.num_envs, max(cfg.num_envs // 8, 1)))[:8] if rank == 0 and not args.no_cpu else []
+    keep = list(range(0, cfg.num_envs, max(cfg.num_envs // CPU_SAMPLE_OBS, 1)))[:CPU_SAMPLE_OBS] if rank == 0 and not args.no_cpu else []
     # the sweep workload moves every camera before every step (seeded walk, pre-computed here)
     walk_steps = args.steps + args.warmup if WORKLOAD == "sweep" else 0
     batch, cams, kept = workload.build_batch(cfg, local, env_offset=shard.env_offset(rank, cfg.num_envs), keep_envs=keep,
@@ -468,7 +471,7 @@ def main():
             rate, n, secs, cores = cpu_oracle_rate(cfg, kept)
             out["cpu_baseline"] = {"value": rate, "unit": "obs/s", "cores": cores, "kind": "oracle", "cpu_model": cpu_model(),
                                    "affinity": cpu_affinity(),
-                                   "sample": f"{n} observations (every {max(cfg.num_envs // 8, 1)}th env) of this workload, all pixels, {secs:.1f} s"}
+                                   "sample": f"{n} observations (every {max(cfg.num_envs // CPU_SAMPLE_OBS, 1)}th env) of this workload, all pixels, {secs:.1f} s"}
         print(json.dumps(out))
     if args.extras and rank == 0:
         print(json.dumps({"extras": time_extras(batch, cfg, cams, rgb, depth, dev)}), file=sys.stderr)

@@ -60,7 +60,7 @@ struct RenderParams {
     uint32_t sky_rgbx;
     float miss_depth;
     int agents_per_cta;                // observations one CTA renders: 1, or all agents of its env
-    int max_steps;                     // bound of the traversal loop: grid_x + grid_y + grid_z + 3
+    int max_steps;                     // most steps a walk can take: grid_x + grid_y + grid_z + 3 (sizes the exit margin)
     float exit_scale;                  // 1 - (bound on the rounding drift of accumulated crossing times)
     // shared-memory offsets after the staged env block: tile table, per-agent blocks (camera record,
     // DDA start table, eye-relative boxes, then overlay rectangles, per-tile box masks and per-tile
