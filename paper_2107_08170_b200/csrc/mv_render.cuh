@@ -131,7 +131,7 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
     " shr.u32 a, pos, 3;\n and.b32 a, a, 0xfffffffc;\n ld.shared.u32 w, [a];\n" MV_DDA_STEP_IDX_TAIL
 #define MV_DDA_STEP_IDX_GLOBAL(T, OUT) MV_DDA_HEAD(T, OUT) MV_DDA_STEP_IDX_ADV \
     " shr.u32 a, pos, 5;\n mad.wide.u32 ag, a, 4, gbase;\n ld.global.nc.u32 w, [ag];\n" MV_DDA_STEP_IDX_TAIL
-// Loop around four steps.  On leaving: ph = a filled cell was entered, thit = when, and px/py
+// Loop around eight steps.  On leaving: ph = a filled cell was entered, thit = when, and px/py
 // still say along which axis.
 #define MV_DDA_LOOP(STEP)                            \
     " setp.ne.u32 pf, 0, 0;\n"                       \
@@ -139,7 +139,8 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
     " mov.f32 tb, 0f00000000;\n"                     \
     "MV_DDA_LOOP_TOP:\n"                             \
     STEP("ta", "MV_DDA_OUT_A") STEP("tb", "MV_DDA_OUT_B") STEP("ta", "MV_DDA_OUT_A") STEP("tb", "MV_DDA_OUT_B") \
-    " sub.s32 it, it, 4;\n"                          \
+    STEP("ta", "MV_DDA_OUT_A") STEP("tb", "MV_DDA_OUT_B") STEP("ta", "MV_DDA_OUT_A") STEP("tb", "MV_DDA_OUT_B") \
+    " sub.s32 it, it, 8;\n"                          \
     " setp.gt.s32 pq, it, 0;\n"                      \
     " @pq bra MV_DDA_LOOP_TOP;\n"                    \
     "MV_DDA_OUT_A:\n"                                \
@@ -491,18 +492,20 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             float t_hit, dtx, dty, dtz;
             if (COLW && cam_in && !MV_BRICKS) {
                 // ---- the common case in one block of PTX: tile record, ray through the pixel centre
-                // (d = F + a*Rs + b*Us, a = 2px+1-W, b = H-1-2py, two chained FMAs per component; a
-                // component that is exactly zero becomes 1e-30 so that it never crosses a cell face and
-                // the slab arithmetic stays finite), reciprocals, the DDA table rows for the ray's signs
+                // (d = F + a*Rs + b*Us, a = 2px+1-W, b = H-1-2py, two chained FMAs per component),
+                // reciprocals, the DDA table rows for the ray's signs
                 // {distance to the first face, cells left, step, colour row} per axis, first crossing
                 // times, exit time, then the walk.  The basis is re-read from shared memory per tile:
                 // three broadcast loads cost less than nine registers held across the walk.
+                // A direction component that is exactly zero needs no special case here: its reciprocal
+                // is +-inf, so its crossing time is +inf (or NaN when the eye sits exactly on the face,
+                // which min and the compares ignore) and that axis is never stepped, which is the rule
+                // for such rays; the exit time ignores the axis the same way.
                 asm volatile("{\n"
                     MV_DDA_DECL
                     " .reg .f32 Ta, Tb, Fx, Fy, Fz, Rx, Ry, Rz, Ux, Uy, Uz, ca, cb, dx, dy, dz, ix, iy, iz;\n"
                     " .reg .f32 q0, q1, q2, q3, q4, q5, esc;\n"
                     " .reg .b32 u, tab;\n"
-                    " .reg .pred p0;\n"
                     " ld.shared.v4.b32 {Ta, Tb, %0, _}, [%9];\n"
                     " ld.shared.f32 Fx, [%10+12];\n"
                     " ld.shared.v4.f32 {Fy, Fz, Rx, Ry}, [%10+16];\n"
@@ -516,12 +519,6 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                     " fma.rn.f32 dx, cb, Ux, dx;\n"
                     " fma.rn.f32 dy, cb, Uy, dy;\n"
                     " fma.rn.f32 dz, cb, Uz, dz;\n"
-                    " setp.eq.f32 p0, dx, 0f00000000;\n"
-                    " selp.f32 dx, 0f0DA24260, dx, p0;\n"
-                    " setp.eq.f32 p0, dy, 0f00000000;\n"
-                    " selp.f32 dy, 0f0DA24260, dy, p0;\n"
-                    " setp.eq.f32 p0, dz, 0f00000000;\n"
-                    " selp.f32 dz, 0f0DA24260, dz, p0;\n"
                     " rcp.approx.ftz.f32 ix, dx;\n"
                     " rcp.approx.ftz.f32 iy, dy;\n"
                     " rcp.approx.ftz.f32 iz, dz;\n"
@@ -733,7 +730,12 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             uint32_t rgbx, m;
             float depth, tb, wmax;
             {
-                const uint32_t vi = COLW ? (pos << 3) + (uint32_t)(31 - __clz(bit)) : pos;
+                uint32_t vi = pos;
+                if (COLW) {
+                    uint32_t y;
+                    asm("bfind.u32 %0, %1;" : "=r"(y) : "r"(bit));
+                    vi = (pos << 3) + y;
+                }
                 asm volatile("{\n"
                     " .reg .pred pv;\n"
                     " .reg .b32 mid, skyb, missb, tbb, wmb;\n"
