@@ -332,7 +332,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     };
     if (tid < kDdaVecs * apc) {
         // DDA start table of agent ag, entry 3*signs + axis (bit c of `signs` set: direction component c
-        // negative): x = signed distance from the eye to the cell face the ray meets first, y = cells
+        // negative): x = distance (>= 0) from the eye to the cell face the ray meets first, y = cells
         // left before the occupied box ends that way, z = what a step along the axis adds to the
         // position (column-word flavour: byte stride for x and z, rotate count for y), w = shared-memory
         // address of the colour-table row of the face entered by a step along this axis.
@@ -350,7 +350,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         int st;
         if (COLW) st = ax == 0 ? (neg ? -4 : 4) : (ax == 1 ? (neg ? 31 : 1) : (neg ? -4 * gx : 4 * gx));
         else st = (ax == 0 ? stride_x : (ax == 1 ? 1 : stride_z)) * (neg ? -1 : 1);
-        agent_dda(ag)[e] = make_float4(neg ? (float)cc - Pc : (float)(cc + 1) - Pc,
+        agent_dda(ag)[e] = make_float4(neg ? Pc - (float)cc : (float)(cc + 1) - Pc,
                                        neg ? (float)(cc - lo_c) : (float)(hi_c - 1 - cc), __int_as_float(st),
                                        __uint_as_float(lut_base + (uint32_t)((2 * ax + neg) * P_ * 4)));
         if (e == 0) {
@@ -519,12 +519,12 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                     " fma.rn.f32 dx, cb, Ux, dx;\n"
                     " fma.rn.f32 dy, cb, Uy, dy;\n"
                     " fma.rn.f32 dz, cb, Uz, dz;\n"
-                    " rcp.approx.ftz.f32 ix, dx;\n"
-                    " rcp.approx.ftz.f32 iy, dy;\n"
-                    " rcp.approx.ftz.f32 iz, dz;\n"
-                    " abs.f32 dtx, ix;\n"
-                    " abs.f32 dty, iy;\n"
-                    " abs.f32 dtz, iz;\n"
+                    " abs.f32 ix, dx;\n"
+                    " abs.f32 iy, dy;\n"
+                    " abs.f32 iz, dz;\n"
+                    " rcp.approx.ftz.f32 dtx, ix;\n"
+                    " rcp.approx.ftz.f32 dty, iy;\n"
+                    " rcp.approx.ftz.f32 dtz, iz;\n"
                     " mov.b32 u, dx;\n"
                     " shr.u32 %8, u, 31;\n"
                     " mov.b32 u, dy;\n"
@@ -537,9 +537,9 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                     " ld.shared.v4.b32 {q0, q1, sx, _}, [tab+" MV_TAB_X "];\n"
                     " ld.shared.v4.b32 {q2, q3, sy, _}, [tab+" MV_TAB_Y "];\n"
                     " ld.shared.v4.b32 {q4, q5, sz, _}, [tab+" MV_TAB_Z "];\n"
-                    " mul.f32 tx, q0, ix;\n"
-                    " mul.f32 ty, q2, iy;\n"
-                    " mul.f32 tz, q4, iz;\n"
+                    " mul.f32 tx, q0, dtx;\n"
+                    " mul.f32 ty, q2, dty;\n"
+                    " mul.f32 tz, q4, dtz;\n"
                     " fma.rn.f32 q1, q1, dtx, tx;\n"
                     " fma.rn.f32 q3, q3, dty, ty;\n"
                     " fma.rn.f32 q5, q5, dtz, tz;\n"
@@ -599,9 +599,9 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                 t_hit = 0.0f;
                 pos = pos0; bit = bit0; row = row0;
                 if (cam_in) {
-                    t0x = qxx * ix;
-                    t0y = qyx * iy;
-                    t0z = qzx * iz;
+                    t0x = qxx * dtx;
+                    t0y = qyx * dty;
+                    t0z = qzx * dtz;
                     t_exit = min3f(fmaf(qxy, dtx, t0x), fmaf(qyy, dty, t0y), fmaf(qzy, dtz, t0z)) * esc;
                 } else {
                     // eye outside the occupied box: clip the ray to it, start in the entry cell
