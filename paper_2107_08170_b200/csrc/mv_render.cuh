@@ -136,7 +136,6 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
 #define MV_DDA_LOOP(STEP)                            \
     " setp.ne.u32 pf, 0, 0;\n"                       \
     " setp.ne.u32 ph, 0, 0;\n"                       \
-    " mov.f32 tb, 0f00000000;\n"                     \
     "MV_DDA_LOOP_TOP:\n"                             \
     STEP("ta", "MV_DDA_OUT_A") STEP("tb", "MV_DDA_OUT_B") STEP("ta", "MV_DDA_OUT_A") STEP("tb", "MV_DDA_OUT_B") \
     STEP("ta", "MV_DDA_OUT_A") STEP("tb", "MV_DDA_OUT_B") STEP("ta", "MV_DDA_OUT_A") STEP("tb", "MV_DDA_OUT_B") \
@@ -177,8 +176,8 @@ constexpr uint32_t kOverlayTileBit = 0x80000000u;   // in a tile's box mask word
 constexpr uint32_t kAgentInside = 1u;      // eye inside the occupied cell box
 constexpr uint32_t kAgentBad = 2u;         // non-finite camera: sky frame
 constexpr uint32_t kAgentFilled = 4u;      // the eye's own voxel is filled
-// Per-agent block in shared memory (16-byte slots): camera record (3), {-, flags, self box, overlay
-// count} (1), {start bit mask, exit-time factor, start colour row, start position} (1), {64-bit address
+// Per-agent block in shared memory (16-byte slots): camera record (3), {hit time a ray starts with,
+// flags, self box, overlay count} (1), {start bit mask, exit-time factor, start colour row, start position} (1), {64-bit address
 // of the env's material store, biased for the walk's positions} (1), DDA start
 // table (8 sign combinations x 3 axes), then eye-relative boxes, overlay rectangles, per-tile box
 // masks and per-tile overlay bits at offsets the host lays out.
@@ -355,6 +354,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                                        __uint_as_float(lut_base + (uint32_t)((2 * ax + neg) * P_ * 4)));
         if (e == 0) {
             const bool filled = cam_in && cell_filled(cx0, cy0, cz0);
+            rec[3].x = filled ? 0.0f : kInf;     // hit time a ray starts with: the eye's own voxel, or none yet
             rec[3].y = __uint_as_float(__float_as_uint(rec[3].y) | (cam_in ? kAgentInside : 0u) | (filled ? kAgentFilled : 0u));
             // exit-time factor: pulls the exit in by the rounding drift of the accumulated crossing
             // times; -inf (the product is then -inf or NaN and the first test ends the walk) when the
@@ -436,21 +436,20 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     const float fhix = (float)hix, fhiy = (float)hiy, fhiz = (float)hiz;
 
     // ---- per-lane constants of the 8 x 4 tile: pixel offsets and the store plan.  Depth goes to the
-    // lane's own pixel; lanes 0..23 each write one 32-bit word (row r, word j) of the tile's four
-    // 24-byte RGB row segments, picked by a byte permute from the packed colours of pixels q0 and
-    // q0+1 of that row.  keep() pins each of them in a register: recomputing them per tile costs
-    // more issue slots than the registers are worth.
+    // lane's own pixel.  A tile row's RGB is 24 bytes = six 32-bit words; word j starts inside pixel
+    // q = j + j/3 of the row (at its byte j % 3) and ends inside pixel q + 1, so the lanes of pixels
+    // 0, 1, 2, 4, 5, 6 of each row write one word each, picked by a byte permute from the lane's own
+    // packed colour and its right neighbour's; the lanes of pixels 3 and 7 store no RGB word.  keep()
+    // pins the constants in registers: recomputing them per tile costs more issue slots than the
+    // registers are worth.
     constexpr int kWarps = NT / 32;
     float lane_a = (float)(2 * (lane & 7)), lane_b = (float)(2 * (lane >> 3));
-    const int st_r = lane / 6, st_j = lane - 6 * st_r;
-    const int st_q0 = (4 * st_j) / 3, st_byte = 4 * st_j - 3 * st_q0;       // first byte within pixel q0
-    uint32_t st_src = (uint32_t)((st_r & 3) * 8 + st_q0);
-    // bytes st_byte.. of pixel q0 (3 of them at most), then pixel q0+1 from its byte 0 (selector 4..)
-    uint32_t st_sel = st_byte == 0 ? 0x4210u : (st_byte == 1 ? 0x5421u : 0x6542u);
-    if (lane >= 24) st_sel = 0xffffffffu;                                   // marks the lanes that store no RGB word
+    const int st_r = lane >> 3, st_q = lane & 7, st_j = st_q - (st_q >> 2), st_byte = st_q & 3;
+    // bytes st_byte.. of the own pixel (3 of them at most), then the neighbour's from its byte 0 (selector 4..)
+    uint32_t st_sel = st_byte == 0 ? 0x4210u : (st_byte == 1 ? 0x5421u : (st_byte == 2 ? 0x6542u : 0xffffffffu));
     const int depth_lane_off = (lane >> 3) * W + (lane & 7);
     const int rgb_lane_off = st_r * W * 3 + st_j * 4;
-    keep(lane_a); keep(lane_b); keep(st_src); keep(st_sel);
+    keep(lane_a); keep(lane_b); keep(st_sel);
     const uint32_t tile_begin = smem_addr(s_tile) + 16u * (uint32_t)warp;
 #if MV_PROBE == 3
     uint32_t tile_end = smem_addr(s_tile);
@@ -485,12 +484,135 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         keep(abase);
         asm volatile("" : "+l"(depth_lane), "+l"(rgb_lane));
 
-        // ---- tiles: warp w takes tiles w, w + nwarps, ... (8 x 4 pixels, one per lane)
-        for (uint32_t tile_p = tile_begin; tile_p < tile_end; tile_p += 16u * kWarps, mask_p += mask_step) {
-            int tile_px;
-            uint32_t pos, bit = 0, row, sgn3;
-            float t_hit, dtx, dty, dtz;
-            if (COLW && cam_in && !MV_BRICKS) {
+        // ---- tiles: warp w takes tiles w, w + nwarps, ... (8 x 4 pixels, one per lane).  Two loops, so
+        // that the choice between the common case and the rest is taken per agent, not per tile; what
+        // follows the walk is the same for both.  The warp-wide reduction and shuffle in it name all 32
+        // lanes, so they wait by themselves for lanes whose walk ran longer.
+        auto finish_tile = [&](uint32_t tile_p, uint32_t mask_p, int tile_px, uint32_t pos, uint32_t bit, uint32_t row,
+                               uint32_t sgn3, float t_hit, float dtx, float dty, float dtz) {
+            // ---- voxel colour (one material byte from global memory, then the shaded table), this
+            // tile's first box-mask word, and the latest voxel hit of the warp (boxes wholly behind it
+            // are skipped).  Predicated, not branched; sky colour and miss depth ride with the material
+            // store's address in the agent block.  (Column-word flavour: the voxel index is rebuilt from
+            // the column's address and the bit.)
+            uint32_t rgbx, m;
+            float depth, tb, wmax;
+            {
+                uint32_t vi = pos;
+                if (COLW) {
+                    uint32_t y;
+                    asm("bfind.u32 %0, %1;" : "=r"(y) : "r"(bit));
+                    vi = (pos << 3) + y;
+                }
+                asm volatile("{\n"
+                    " .reg .pred pv;\n"
+                    " .reg .b32 mid, skyb, missb, tbb, wmb;\n"
+                    " .reg .b64 mp, sm;\n"
+                    " ld.shared.v2.b64 {mp, sm}, [%8+80];\n"
+                    " ld.shared.u32 %2, [%9];\n"
+                    " mov.b64 {skyb, missb}, sm;\n"
+                    " mov.b32 %0, skyb;\n"
+                    " mov.b32 %1, missb;\n"
+                    " setp.ne.u32 pv, %5, 0xffffffff;\n"
+                    " mad.wide.u32 mp, %6, 1, mp;\n"
+                    " mov.b32 tbb, %7;\n"
+                    " @pv ld.global.nc.u8 mid, [mp];\n"
+                    " @pv mad.lo.u32 mid, mid, 4, %5;\n"
+                    " redux.sync.max.u32 wmb, tbb, 0xffffffff;\n"
+                    " mov.b32 %3, tbb;\n"
+                    " mov.b32 %4, wmb;\n"
+                    " @pv ld.shared.u32 %0, [mid];\n"
+                    " @pv mov.f32 %1, %7;\n"
+                    "}\n"
+                    : "=&r"(rgbx), "=&f"(depth), "=&r"(m), "=&f"(tb), "=&f"(wmax)
+                    : "r"(row), "r"(vi), "f"(t_hit), "r"(abase), "r"(mask_p)
+                    : "memory");
+            }
+#if MV_PROBE == 9
+            depth = t_hit;
+#endif
+#if MV_PROBE >= 2 && MV_PROBE < 9
+            m = 0;
+#endif
+
+            // ---- the less common work, behind one test: boxes binned to this tile (or more than 32 boxes
+            // per environment) and the GUI overlay.  A box wins only with a strictly smaller time.
+            if ((m | rare) != 0u) {
+                if (p.max_boxes < 32) m &= ~kOverlayTileBit;
+                if (m != 0u || mw > 1) {
+                    // signed reciprocals again, and the ray's rows of the DDA table for the faces
+                    const float ix = __uint_as_float(__float_as_uint(dtx) | (sgn3 << 31));
+                    const float iy = __uint_as_float(__float_as_uint(dty) | ((sgn3 & 2u) << 30));
+                    const float iz = __uint_as_float(__float_as_uint(dtz) | ((sgn3 & 4u) << 29));
+                    const uint32_t tab = abase + 48u * sgn3;
+                    uint32_t baddr = 0;
+                    for (int w = 0;;) {
+                        while (m) {
+                            const int b = (__ffs(m) - 1) + 32 * w;
+                            m &= m - 1;
+                            float4 lo, hi;
+                            const uint32_t rel_p = abase + kAgentRelOff + 32u * (uint32_t)b;
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(lo.x), "=f"(lo.y), "=f"(lo.z), "=f"(lo.w) : "r"(rel_p));
+                            if (lo.w > wmax) continue;
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4+16];" : "=f"(hi.x), "=f"(hi.y), "=f"(hi.z), "=f"(hi.w) : "r"(rel_p));
+                            const float x1 = lo.x * ix, x2 = hi.x * ix, y1 = lo.y * iy, y2 = hi.y * iy;
+                            const float z1 = lo.z * iz, z2 = hi.z * iz;
+                            const float nx = fminf(x1, x2), ny = fminf(y1, y2), nz = fminf(z1, z2);
+                            const float tn = max3f(nx, ny, nz);
+                            const float tf = min3f(fmaxf(x1, x2), fmaxf(y1, y2), fmaxf(z1, z2));
+                            const float t = fmaxf(tn, 0.0f);
+                            if ((tn <= tf) && (tf > 0.0f) && (t < tb)) {
+                                tb = t;
+                                uint32_t r = inside_row;
+                                if (!(tn < 0.0f))
+                                    asm volatile("ld.shared.u32 %0, [%1+" MV_TAB_ROW "];" : "=r"(r)
+                                                 : "r"(tab + ((nx == tn) ? 0u : ((ny == tn) ? 16u : 32u))));
+                                baddr = r + 4u * __float_as_uint(hi.w);
+                            }
+                        }
+                        if (++w >= mw) break;
+                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(m) : "r"(mask_p + 4u * (uint32_t)w));
+                    }
+                    if (baddr) {
+                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(rgbx) : "r"(baddr));
+                        depth = tb + 0.0f;
+                    }
+                }
+                // GUI overlay: rectangles in list order, later ones on top; depth is left alone
+                if (ov_count > 0) {
+                    const uint32_t tile_no = (tile_p - smem_addr(s_tile)) >> 4;
+                    if ((agent_ovtile(ag)[tile_no >> 5] >> (tile_no & 31)) & 1u) {
+                        const int4 *ov = agent_ov(ag);
+                        const int px = (tile_px % W) + (lane & 7), py = (tile_px / W) + (lane >> 3);
+                        for (int r = 0; r < ov_count; ++r) {
+                            const int4 q = ov[2 * r];
+                            if (px >= q.x && px < q.z && py >= q.y && py < q.w) rgbx = (uint32_t)ov[2 * r + 1].x;
+                        }
+                    }
+                }
+            }
+
+            // ---- store: depth rows are 32-byte segments; RGB rows are 24 bytes = 6 packed words
+            asm volatile("{\n"
+                " .reg .pred ps;\n"
+                " .reg .b32 ca, cb;\n"
+                " .reg .b64 ad;\n"
+                " mad.wide.s32 ad, %2, 4, %3;\n"
+                " st.global.f32 [ad], %1;\n"
+                " shfl.sync.down.b32 cb, %0, 1, 31, 0xffffffff;\n"
+                " mad.wide.s32 ad, %2, 3, %4;\n"
+                " prmt.b32 ca, %0, cb, %5;\n"
+                " setp.ge.s32 ps, %5, 0;\n"
+                " @ps st.global.u32 [ad], ca;\n"
+                "}\n"
+                :: "r"(rgbx), "f"(depth), "r"(tile_px), "l"(depth_lane), "l"(rgb_lane), "r"(st_sel)
+                : "memory");
+        };
+        if (COLW && cam_in && !MV_BRICKS) {
+            for (uint32_t tile_p = tile_begin; tile_p < tile_end; tile_p += 16u * kWarps, mask_p += mask_step) {
+                int tile_px;
+                uint32_t pos, bit = 0, row, sgn3;
+                float t_hit, dtx, dty, dtz;
                 // ---- the common case in one block of PTX: tile record, ray through the pixel centre
                 // (d = F + a*Rs + b*Us, a = 2px+1-W, b = H-1-2py, two chained FMAs per component),
                 // reciprocals, the DDA table rows for the ray's signs
@@ -548,13 +670,12 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
 #if MV_PROBE >= 1 && MV_PROBE < 9
                     " mov.f32 texit, 0fFF800000;\n"
 #endif
-                    " mov.f32 thit, 0f00000000;\n"
+                    " ld.shared.f32 thit, [%10+48];\n"
                     " mov.s32 it, " MV_STEP_BUDGET ";\n"
                     MV_DDA_LOOP(MV_DDA_STEP_COLW)
-                    " selp.u32 a, 16, 32, py;\n"
-                    " selp.u32 a, 0, a, px;\n"
-                    " add.u32 a, a, tab;\n"
-                    " @ph ld.shared.u32 %4, [a+" MV_TAB_ROW "];\n"
+                    " @py add.u32 tab, tab, 16;\n"
+                    " @pz add.u32 tab, tab, 32;\n"
+                    " @ph ld.shared.u32 %4, [tab+" MV_TAB_ROW "];\n"
 #if MV_PROBE == 9
                     " mov.f32 thit, ns;\n"
 #endif
@@ -568,7 +689,13 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                     : "=&r"(tile_px), "=&r"(pos), "=&r"(bit), "=&f"(t_hit), "=&r"(row), "=&f"(dtx), "=&f"(dty), "=&f"(dtz), "=&r"(sgn3)
                     : "r"(tile_p), "r"(abase), "f"(lane_a), "f"(lane_b)
                     : "memory");
-            } else {
+                finish_tile(tile_p, mask_p, tile_px, pos, bit, row, sgn3, t_hit, dtx, dty, dtz);
+            }
+        } else {
+            for (uint32_t tile_p = tile_begin; tile_p < tile_end; tile_p += 16u * kWarps, mask_p += mask_step) {
+                int tile_px;
+                uint32_t pos, bit = 0, row, sgn3;
+                float t_hit, dtx, dty, dtz;
                 // ---- every other case: the same steps in C++, with the eye possibly outside the
                 // occupied box and either flavour of the walk
                 float Ta, Tb;
@@ -719,130 +846,9 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
 #undef MV_DDA_IO
 #undef MV_DDA_IN
 #undef MV_DDA_OUTS
+                if (row == kNoRow) t_hit = kInf;          // no voxel hit
+                finish_tile(tile_p, mask_p, tile_px, pos, bit, row, sgn3, t_hit, dtx, dty, dtz);
             }
-            __syncwarp();
-
-            // ---- voxel colour (one material byte from global memory, then the shaded table), this
-            // tile's first box-mask word, and the latest voxel hit of the warp (boxes wholly behind it
-            // are skipped).  Predicated, not branched; sky colour and miss depth ride with the material
-            // store's address in the agent block.  (Column-word flavour: the voxel index is rebuilt from
-            // the column's address and the bit.)
-            uint32_t rgbx, m;
-            float depth, tb, wmax;
-            {
-                uint32_t vi = pos;
-                if (COLW) {
-                    uint32_t y;
-                    asm("bfind.u32 %0, %1;" : "=r"(y) : "r"(bit));
-                    vi = (pos << 3) + y;
-                }
-                asm volatile("{\n"
-                    " .reg .pred pv;\n"
-                    " .reg .b32 mid, skyb, missb, tbb, wmb;\n"
-                    " .reg .b64 mp, sm;\n"
-                    " ld.shared.v2.b64 {mp, sm}, [%8+80];\n"
-                    " ld.shared.u32 %2, [%9];\n"
-                    " mov.b64 {skyb, missb}, sm;\n"
-                    " mov.b32 %0, skyb;\n"
-                    " mov.b32 %1, missb;\n"
-                    " setp.ne.u32 pv, %5, 0xffffffff;\n"
-                    " cvt.u64.u32 sm, %6;\n"
-                    " add.u64 mp, mp, sm;\n"
-                    " mov.b32 tbb, 0x7F800000;\n"
-                    " @pv ld.global.nc.u8 mid, [mp];\n"
-                    " @pv mov.b32 tbb, %7;\n"
-                    " @pv mad.lo.u32 mid, mid, 4, %5;\n"
-                    " redux.sync.max.u32 wmb, tbb, 0xffffffff;\n"
-                    " mov.b32 %3, tbb;\n"
-                    " mov.b32 %4, wmb;\n"
-                    " @pv ld.shared.u32 %0, [mid];\n"
-                    " @pv mov.f32 %1, %7;\n"
-                    "}\n"
-                    : "=&r"(rgbx), "=&f"(depth), "=&r"(m), "=&f"(tb), "=&f"(wmax)
-                    : "r"(row), "r"(vi), "f"(t_hit), "r"(abase), "r"(mask_p)
-                    : "memory");
-            }
-#if MV_PROBE == 9
-            depth = t_hit;
-#endif
-#if MV_PROBE >= 2 && MV_PROBE < 9
-            m = 0;
-#endif
-
-            // ---- the less common work, behind one test: boxes binned to this tile (or more than 32 boxes
-            // per environment) and the GUI overlay.  A box wins only with a strictly smaller time.
-            if ((m | rare) != 0u) {
-                if (p.max_boxes < 32) m &= ~kOverlayTileBit;
-                if (m != 0u || mw > 1) {
-                    // signed reciprocals again, and the ray's rows of the DDA table for the faces
-                    const float ix = __uint_as_float(__float_as_uint(dtx) | (sgn3 << 31));
-                    const float iy = __uint_as_float(__float_as_uint(dty) | ((sgn3 & 2u) << 30));
-                    const float iz = __uint_as_float(__float_as_uint(dtz) | ((sgn3 & 4u) << 29));
-                    const uint32_t tab = abase + 48u * sgn3;
-                    uint32_t baddr = 0;
-                    for (int w = 0;;) {
-                        while (m) {
-                            const int b = (__ffs(m) - 1) + 32 * w;
-                            m &= m - 1;
-                            float4 lo, hi;
-                            const uint32_t rel_p = abase + kAgentRelOff + 32u * (uint32_t)b;
-                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(lo.x), "=f"(lo.y), "=f"(lo.z), "=f"(lo.w) : "r"(rel_p));
-                            if (lo.w > wmax) continue;
-                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4+16];" : "=f"(hi.x), "=f"(hi.y), "=f"(hi.z), "=f"(hi.w) : "r"(rel_p));
-                            const float x1 = lo.x * ix, x2 = hi.x * ix, y1 = lo.y * iy, y2 = hi.y * iy;
-                            const float z1 = lo.z * iz, z2 = hi.z * iz;
-                            const float nx = fminf(x1, x2), ny = fminf(y1, y2), nz = fminf(z1, z2);
-                            const float tn = max3f(nx, ny, nz);
-                            const float tf = min3f(fmaxf(x1, x2), fmaxf(y1, y2), fmaxf(z1, z2));
-                            const float t = fmaxf(tn, 0.0f);
-                            if ((tn <= tf) && (tf > 0.0f) && (t < tb)) {
-                                tb = t;
-                                uint32_t r = inside_row;
-                                if (!(tn < 0.0f))
-                                    asm volatile("ld.shared.u32 %0, [%1+" MV_TAB_ROW "];" : "=r"(r)
-                                                 : "r"(tab + ((nx == tn) ? 0u : ((ny == tn) ? 16u : 32u))));
-                                baddr = r + 4u * __float_as_uint(hi.w);
-                            }
-                        }
-                        if (++w >= mw) break;
-                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(m) : "r"(mask_p + 4u * (uint32_t)w));
-                    }
-                    if (baddr) {
-                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(rgbx) : "r"(baddr));
-                        depth = tb + 0.0f;
-                    }
-                }
-                // GUI overlay: rectangles in list order, later ones on top; depth is left alone
-                if (ov_count > 0) {
-                    const uint32_t tile_no = (tile_p - smem_addr(s_tile)) >> 4;
-                    if ((agent_ovtile(ag)[tile_no >> 5] >> (tile_no & 31)) & 1u) {
-                        const int4 *ov = agent_ov(ag);
-                        const int px = (tile_px % W) + (lane & 7), py = (tile_px / W) + (lane >> 3);
-                        for (int r = 0; r < ov_count; ++r) {
-                            const int4 q = ov[2 * r];
-                            if (px >= q.x && px < q.z && py >= q.y && py < q.w) rgbx = (uint32_t)ov[2 * r + 1].x;
-                        }
-                    }
-                }
-            }
-
-            // ---- store: depth rows are 32-byte segments; RGB rows are 24 bytes = 6 packed words
-            asm volatile("{\n"
-                " .reg .pred ps;\n"
-                " .reg .b32 ca, cb, s2;\n"
-                " .reg .b64 ad;\n"
-                " mad.wide.s32 ad, %2, 4, %3;\n"
-                " st.global.f32 [ad], %1;\n"
-                " shfl.sync.idx.b32 ca, %0, %5, 31, 0xffffffff;\n"
-                " add.u32 s2, %5, 1;\n"
-                " shfl.sync.idx.b32 cb, %0, s2, 31, 0xffffffff;\n"
-                " mad.wide.s32 ad, %2, 3, %4;\n"
-                " prmt.b32 ca, ca, cb, %6;\n"
-                " setp.ge.s32 ps, %6, 0;\n"
-                " @ps st.global.u32 [ad], ca;\n"
-                "}\n"
-                :: "r"(rgbx), "f"(depth), "r"(tile_px), "l"(depth_lane), "l"(rgb_lane), "r"(st_src), "r"(st_sel)
-                : "memory");
         }
     }
 }
