@@ -247,21 +247,26 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         bulk_load(smem, env_block + unstaged, p.lay.block_bytes - unstaged, s_bar);
     }
     // ---- meanwhile: tile table, cleared masks, camera records, GUI rectangles
-    for (int i = tid; i < apc * ntiles * mw; i += NT) agent_mask(i / (ntiles * mw))[i % (ntiles * mw)] = 0u;
+    for (int ag = 0; ag < apc; ++ag) {
+        uint32_t *mk = agent_mask(ag);
+        for (int i = tid; i < ntiles * mw; i += NT) mk[i] = 0u;
+    }
+    const float inv_tiles_x = 1.0f / (float)p.tiles_x;
     for (int i = tid; i < ntiles; i += NT) {
-        const int ty = i / p.tiles_x, tx = i - ty * p.tiles_x;
+        // (i + 0.5) / tiles_x is at least 1 / (2 tiles_x) away from an integer: exact in float for any image
+        const int ty = (int)(((float)i + 0.5f) * inv_tiles_x), tx = i - ty * p.tiles_x;
         // a = 2px+1-W and b = H-1-2py of the tile's first pixel (small integers: exact as floats)
         s_tile[i] = make_float4((float)(16 * tx + 1 - W), (float)(H - 1 - 8 * ty), __int_as_float(ty * 4 * W + tx * 8),
                                 __int_as_float(i));
     }
-    if (tid < apc) {
-        const float4 *cq = reinterpret_cast<const float4 *>(p.cams + obs0 + tid);
+    for (int ag = tid; ag < apc; ag += NT) {
+        const float4 *cq = reinterpret_cast<const float4 *>(p.cams + obs0 + ag);
         const float4 c3 = __ldg(cq + 3);
-        float4 *rec = agent_rec(tid);
+        float4 *rec = agent_rec(ag);
         rec[0] = __ldg(cq);
         rec[1] = __ldg(cq + 1);
         rec[2] = __ldg(cq + 2);
-        const int ovc = p.overlay ? min(max(__ldg(p.overlay_count + obs0 + tid), 0), p.max_overlay) : 0;
+        const int ovc = p.overlay ? min(max(__ldg(p.overlay_count + obs0 + ag), 0), p.max_overlay) : 0;
         rec[3] = make_float4(0.0f, __uint_as_float((__float_as_uint(c3.y) & kFlagBadCamera) ? kAgentBad : 0u), c3.x,
                              __int_as_float(ovc));
     }
@@ -329,13 +334,13 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         const uint32_t u = (uint32_t)(stride_x * cx + stride_z * cz + cy);
         return (s_occ[u >> 5] >> (u & 31)) & 1u;
     };
-    if (tid < kDdaVecs * apc) {
+    for (int slot = tid; slot < kDdaVecs * apc; slot += NT) {
         // DDA start table of agent ag, entry 3*signs + axis (bit c of `signs` set: direction component c
         // negative): x = distance (>= 0) from the eye to the cell face the ray meets first, y = cells
         // left before the occupied box ends that way, z = what a step along the axis adds to the
         // position (column-word flavour: byte stride for x and z, rotate count for y), w = shared-memory
         // address of the colour-table row of the face entered by a step along this axis.
-        const int ag = tid / kDdaVecs, e = tid - ag * kDdaVecs;
+        const int ag = slot / kDdaVecs, e = slot - ag * kDdaVecs;
         const int signs = e / 3, ax = e - 3 * signs, neg = (signs >> ax) & 1;
         float4 *rec = agent_rec(ag);
         const float4 c0 = rec[0];

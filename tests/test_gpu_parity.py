@@ -482,6 +482,31 @@ def test_cta_per_environment_equals_cta_per_observation():
     batch.destroy()
 
 
+def test_twenty_agents_in_one_cta(oracle):
+    """More agents per CTA than one pass of the CTA's threads over the per-agent set-up covers
+    (20 x 24 table slots > 384 threads): every agent's frame must still equal the per-observation
+    shape's, and the oracle's."""
+    from gpu_util import upload_scene, scene_to_numpy
+    B = _binding()
+    cfg = scenes.config("tiny", num_envs=3, agents=20, seed=77)
+    sc = scenes.make_scene(cfg)
+    batch = B.Batch(B.desc_from_config(cfg))
+    upload_scene(batch, sc)
+    batch.set_cameras(sc["cams"].cuda().contiguous())
+    out = {}
+    for apc in (1, cfg.agents):
+        batch.debug_agents_per_cta(apc)
+        rgb, depth = batch.alloc_outputs()
+        rgb.fill_(9); depth.fill_(-3.0)
+        batch.render_batch(rgb, depth)
+        assert batch.query_status() == 0
+        out[apc] = (rgb.cpu(), depth.cpu())
+    assert torch.equal(out[1][0], out[20][0]) and torch.equal(out[1][1], out[20][1])
+    st = parity.compare_scene(oracle, cfg, scene_to_numpy(sc), range(cfg.num_obs), out[20][0].numpy(), out[20][1].numpy())
+    parity.assert_parity(st, "20 agents per CTA")
+    batch.destroy()
+
+
 def test_two_batches_of_different_shape_alive_together():
     """The kernel's shared-memory cap is per function and device, not per batch: a small batch created
     after a large one must not make the large one's launch fail."""
