@@ -374,7 +374,9 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     }
     {
         const int nb = min(s_count[0], p.max_boxes);
-        for (int i = tid; i < apc * p.max_boxes; i += NT) {
+        // (dealt from the last thread down, so that the warps that build the DDA tables above are not
+        // the ones that bin the boxes)
+        for (int i = NT - 1 - tid; i < apc * p.max_boxes; i += NT) {
             const int ag = i / p.max_boxes, b = i - ag * p.max_boxes;
             const float4 *rec = agent_rec(ag);
             const float4 c0 = rec[0], c1 = rec[1], c2 = rec[2];
