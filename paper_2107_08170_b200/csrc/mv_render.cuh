@@ -853,7 +853,9 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
 #undef MV_DDA_IO
 #undef MV_DDA_IN
 #undef MV_DDA_OUTS
+#if MV_PROBE != 9
                 if (row == kNoRow) t_hit = kInf;          // no voxel hit
+#endif
                 finish_tile(tile_p, mask_p, tile_px, pos, bit, row, sgn3, t_hit, dtx, dty, dtz);
             }
         }
