@@ -150,6 +150,21 @@ int mv_upload_worlds(mv_batch *batch, int env_begin, int env_count, const uint8_
                      const mv_box *d_boxes, const int32_t *d_box_count, const uint8_t *d_palette,
                      void *cuda_stream);
 
+/* The same upload for envs that are not neighbours (paper Appendix A.1: environments end their
+ * episodes at different steps and are reset on their own): env i of the arrays goes to env
+ * h_env_index[i] of the batch.
+ *   h_env_index HOST int32 [env_count], strictly increasing, each in [0, num_envs).  It is copied to
+ *               the device in stream order; if it lies in pinned memory the caller keeps it unchanged
+ *               until the stream has passed this call.  The batch owns one device buffer for it, so
+ *               scattered uploads of one batch go to one stream at a time.
+ *   the other arguments: as for mv_upload_worlds, indexed by i.
+ * No counterpart in the paper's interface (its environments reset inside the simulator).
+ * Errors: INVALID_ARG (null list, index out of range or not increasing, d_boxes without
+ * d_box_count), CUDA. */
+int mv_upload_worlds_at(mv_batch *batch, int env_count, const int32_t *h_env_index, const uint8_t *d_grid,
+                        const mv_box *d_boxes, const int32_t *d_box_count, const uint8_t *d_palette,
+                        void *cuda_stream);
+
 /* Set all cameras (paper Section 3.2: cameras are part of the state; Appendix A.1: N x M
  * observations per step) and build each one's ray basis on the device.
  *   d_cams DEVICE mv_camera [num_envs*agents_per_env]

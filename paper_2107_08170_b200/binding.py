@@ -15,7 +15,7 @@ _lib = None
 
 MV_OK = 0
 FLAG_MATERIAL_CLAMPED, FLAG_BOX_COUNT_CLAMPED, FLAG_BAD_CAMERA, FLAG_DEVICE_TIMEOUT = 1, 2, 4, 8
-EXPORTS = ["mv_create_batch", "mv_upload_worlds", "mv_set_cameras", "mv_render_batch", "mv_step_host",
+EXPORTS = ["mv_create_batch", "mv_upload_worlds", "mv_upload_worlds_at", "mv_set_cameras", "mv_render_batch", "mv_step_host",
            "mv_step_host_static", "mv_set_overlays", "mv_move_agents", "mv_merge_voxels", "mv_debug_staging", "mv_debug_occupancy_in_global", "mv_debug_agents_per_cta", "mv_query_status", "mv_launch_count", "mv_destroy", "mv_status_string"]
 
 
@@ -45,6 +45,7 @@ def lib() -> C.CDLL:
         vp, i = C.c_void_p, C.c_int
         L.mv_create_batch.argtypes = [C.POINTER(BatchDesc), C.POINTER(vp)]
         L.mv_upload_worlds.argtypes = [vp, i, i, vp, vp, vp, vp, vp]
+        L.mv_upload_worlds_at.argtypes = [vp, i, vp, vp, vp, vp, vp, vp]
         L.mv_set_cameras.argtypes = [vp, vp, vp]
         L.mv_render_batch.argtypes = [vp, vp, vp, vp]
         L.mv_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -145,6 +146,14 @@ class Batch:
         _check(lib().mv_upload_worlds(self._h, env_begin, env_count, _dptr(grid, torch.uint8),
                                       _dptr(boxes, torch.int32), _dptr(box_count, torch.int32),
                                       _dptr(palette, torch.uint8), _stream(stream)), "mv_upload_worlds")
+
+    def upload_worlds_at(self, env_index, grid=None, boxes=None, box_count=None, palette=None, stream=None):
+        """env_index: strictly increasing env numbers (any int sequence or CPU tensor); the arrays hold
+        one entry per listed env."""
+        idx = torch.as_tensor(env_index, dtype=torch.int32, device="cpu").contiguous()
+        _check(lib().mv_upload_worlds_at(self._h, idx.numel(), C.c_void_p(idx.data_ptr()), _dptr(grid, torch.uint8),
+                                         _dptr(boxes, torch.int32), _dptr(box_count, torch.int32),
+                                         _dptr(palette, torch.uint8), _stream(stream)), "mv_upload_worlds_at")
 
     def set_cameras(self, cams, stream=None):
         _check(lib().mv_set_cameras(self._h, _dptr(cams, torch.int32), _stream(stream)), "mv_set_cameras")

@@ -42,6 +42,7 @@ struct mv_batch {
     int merge_chunk = 0;
     int4 *d_overlay = nullptr;          // [O][max_overlay_rects]
     int32_t *d_overlay_count = nullptr; // [O]
+    int32_t *d_env_index = nullptr;     // [E] destination envs of a scattered upload (mv_upload_worlds_at)
     // host-side readiness tracking (per env)
     std::vector<uint8_t> has_grid, has_palette;
     int missing_grid = 0, missing_palette = 0;
@@ -177,11 +178,11 @@ int launch_cameras(mv_batch *b, const mv_camera *d_cams, cudaStream_t s) {
     return MV_OK;
 }
 
-int launch_boxes(mv_batch *b, int env_begin, int env_count, const mv_box *d_boxes, const int32_t *d_count,
-                 cudaStream_t s) {
+int launch_boxes(mv_batch *b, int env_begin, const int32_t *d_env_index, int env_count, const mv_box *d_boxes,
+                 const int32_t *d_count, cudaStream_t s) {
     const int n = env_count * (b->desc.max_boxes + 1);
     copy_boxes_kernel<<<(n + 255) / 256, 256, 0, s>>>(reinterpret_cast<const uint4 *>(d_boxes), d_count,
-                                                       b->d_env_blocks, b->lay, env_begin, env_count,
+                                                       b->d_env_blocks, b->lay, env_begin, d_env_index, env_count,
                                                        b->desc.max_boxes, b->desc.palette_size, b->d_status);
     b->launches++;
     MV_CUDA(b, cudaGetLastError());
@@ -257,6 +258,64 @@ int static_scratch_for_device(mv_batch *b, int device, unsigned char **out) {
         g_static_scratch_ptr[device] = static_cast<unsigned char *>(p);
     }
     *out = g_static_scratch_ptr[device];
+    return MV_OK;
+}
+}  // namespace
+
+namespace {
+// Body of both upload entry points.  h_env_index: null for the contiguous range that starts at
+// env_begin, else the (validated) destination env of each uploaded env.
+int upload_worlds(mv_batch *b, int env_begin, const int32_t *h_env_index, int env_count, const uint8_t *d_grid,
+                  const mv_box *d_boxes, const int32_t *d_box_count, const uint8_t *d_palette, cudaStream_t s) {
+    if (d_boxes && !d_box_count) return MV_ERR_INVALID_ARG;
+    if (d_boxes && b->desc.max_boxes == 0) return MV_ERR_INVALID_ARG;
+    if ((d_grid && !aligned16(d_grid)) || (d_boxes && !aligned16(d_boxes))) return MV_ERR_INVALID_ARG;
+    if (env_count == 0) return MV_OK;
+    DeviceGuard g(b->desc.device);
+    if (!g.ok) return MV_ERR_CUDA;
+    const int32_t *d_index = nullptr;
+    if (h_env_index) {
+        // The list is copied in stream order into a buffer the batch owns; an earlier scattered upload
+        // on another stream that has not finished would be overwritten (one stream at a time).
+        MV_CUDA(b, cudaMemcpyAsync(b->d_env_index, h_env_index, (size_t)env_count * 4, cudaMemcpyHostToDevice, s));
+        d_index = b->d_env_index;
+    }
+    auto dst_env = [&](int i) { return h_env_index ? h_env_index[i] : env_begin + i; };
+    if (d_grid) {
+        const size_t threads = ((size_t)(b->desc.grid_x / 4) * b->desc.grid_z << (b->lay.ysh - 5)) * (size_t)env_count;
+        const size_t blocks = (threads + 255) / 256;
+        if (blocks > 0x7fffffffull) return MV_ERR_INVALID_ARG;
+        pack_grid_kernel<<<(unsigned)blocks, 256, 0, s>>>(d_grid, b->d_env_blocks, b->d_mat, b->lay, b->desc.grid_x,
+                                                           b->desc.grid_y, b->desc.grid_z, env_begin, d_index, env_count,
+                                                           b->desc.palette_size, b->d_status);
+        b->launches++;
+        MV_CUDA(b, cudaGetLastError());
+        occupied_bounds_kernel<<<env_count, 256, 0, s>>>(b->d_env_blocks, b->lay, env_begin, d_index, b->desc.grid_x,
+                                                          b->desc.grid_y, b->desc.grid_z);
+        b->launches++;
+        MV_CUDA(b, cudaGetLastError());
+        for (int i = 0; i < env_count; ++i) {
+            const int e = dst_env(i);
+            if (!b->has_grid[e]) { b->has_grid[e] = 1; b->missing_grid--; }
+        }
+    }
+    if (d_palette) {
+        const int n = env_count * kFaces * b->desc.palette_size;
+        build_lut_kernel<<<(n + 255) / 256, 256, 0, s>>>(d_palette, b->d_env_blocks, b->lay, env_begin, d_index, env_count,
+                                                          b->desc.palette_size, (double)b->desc.light_dir[0],
+                                                          (double)b->desc.light_dir[1], (double)b->desc.light_dir[2],
+                                                          (double)b->desc.ambient);
+        b->launches++;
+        MV_CUDA(b, cudaGetLastError());
+        for (int i = 0; i < env_count; ++i) {
+            const int e = dst_env(i);
+            if (!b->has_palette[e]) { b->has_palette[e] = 1; b->missing_palette--; }
+        }
+    }
+    if (d_boxes) {
+        int r = launch_boxes(b, env_begin, d_index, env_count, d_boxes, d_box_count, s);
+        if (r != MV_OK) return r;
+    }
     return MV_OK;
 }
 }  // namespace
@@ -370,7 +429,8 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
     bool ok = cudaMalloc(&b->d_env_blocks, blocks_bytes) == cudaSuccess &&
               cudaMalloc(&b->d_mat, (size_t)d.num_envs * b->mat_bytes_per_env) == cudaSuccess &&
               cudaMalloc(&b->d_cams, (size_t)b->num_obs * sizeof(CamRec)) == cudaSuccess &&
-              cudaMalloc(&b->d_status, 16) == cudaSuccess;
+              cudaMalloc(&b->d_status, 16) == cudaSuccess &&
+              cudaMalloc(&b->d_env_index, (size_t)d.num_envs * 4) == cudaSuccess;
     if (ok && d.max_overlay_rects > 0)
         ok = cudaMalloc(&b->d_overlay, (size_t)b->num_obs * d.max_overlay_rects * 16) == cudaSuccess &&
              cudaMalloc(&b->d_overlay_count, (size_t)b->num_obs * 4) == cudaSuccess &&
@@ -390,45 +450,20 @@ int mv_upload_worlds(mv_batch *b, int env_begin, int env_count, const uint8_t *d
                      const int32_t *d_box_count, const uint8_t *d_palette, void *cuda_stream) {
     if (!b || env_begin < 0 || env_count < 0 || (int64_t)env_begin + env_count > b->desc.num_envs)
         return MV_ERR_INVALID_ARG;
-    if (d_boxes && !d_box_count) return MV_ERR_INVALID_ARG;
-    if (d_boxes && b->desc.max_boxes == 0) return MV_ERR_INVALID_ARG;
-    if ((d_grid && !aligned16(d_grid)) || (d_boxes && !aligned16(d_boxes))) return MV_ERR_INVALID_ARG;
-    if (env_count == 0) return MV_OK;
-    DeviceGuard g(b->desc.device);
-    if (!g.ok) return MV_ERR_CUDA;
-    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (d_grid) {
-        const size_t threads = ((size_t)(b->desc.grid_x / 4) * b->desc.grid_z << (b->lay.ysh - 5)) * (size_t)env_count;
-        const size_t blocks = (threads + 255) / 256;
-        if (blocks > 0x7fffffffull) return MV_ERR_INVALID_ARG;
-        pack_grid_kernel<<<(unsigned)blocks, 256, 0, s>>>(d_grid, b->d_env_blocks, b->d_mat, b->lay, b->desc.grid_x,
-                                                           b->desc.grid_y, b->desc.grid_z, env_begin, env_count,
-                                                           b->desc.palette_size, b->d_status);
-        b->launches++;
-        MV_CUDA(b, cudaGetLastError());
-        occupied_bounds_kernel<<<env_count, 256, 0, s>>>(b->d_env_blocks, b->lay, env_begin, b->desc.grid_x,
-                                                          b->desc.grid_y, b->desc.grid_z);
-        b->launches++;
-        MV_CUDA(b, cudaGetLastError());
-        for (int e = env_begin; e < env_begin + env_count; ++e)
-            if (!b->has_grid[e]) { b->has_grid[e] = 1; b->missing_grid--; }
-    }
-    if (d_palette) {
-        const int n = env_count * kFaces * b->desc.palette_size;
-        build_lut_kernel<<<(n + 255) / 256, 256, 0, s>>>(d_palette, b->d_env_blocks, b->lay, env_begin, env_count,
-                                                          b->desc.palette_size, (double)b->desc.light_dir[0],
-                                                          (double)b->desc.light_dir[1], (double)b->desc.light_dir[2],
-                                                          (double)b->desc.ambient);
-        b->launches++;
-        MV_CUDA(b, cudaGetLastError());
-        for (int e = env_begin; e < env_begin + env_count; ++e)
-            if (!b->has_palette[e]) { b->has_palette[e] = 1; b->missing_palette--; }
-    }
-    if (d_boxes) {
-        int r = launch_boxes(b, env_begin, env_count, d_boxes, d_box_count, s);
-        if (r != MV_OK) return r;
-    }
-    return MV_OK;
+    return upload_worlds(b, env_begin, nullptr, env_count, d_grid, d_boxes, d_box_count, d_palette,
+                         static_cast<cudaStream_t>(cuda_stream));
+}
+
+int mv_upload_worlds_at(mv_batch *b, int env_count, const int32_t *h_env_index, const uint8_t *d_grid,
+                        const mv_box *d_boxes, const int32_t *d_box_count, const uint8_t *d_palette,
+                        void *cuda_stream) {
+    if (!b || env_count < 0 || env_count > b->desc.num_envs || (env_count > 0 && !h_env_index))
+        return MV_ERR_INVALID_ARG;
+    for (int i = 0; i < env_count; ++i)          // strictly increasing: in range and no env written twice
+        if (h_env_index[i] < 0 || h_env_index[i] >= b->desc.num_envs || (i > 0 && h_env_index[i] <= h_env_index[i - 1]))
+            return MV_ERR_INVALID_ARG;
+    return upload_worlds(b, 0, h_env_index, env_count, d_grid, d_boxes, d_box_count, d_palette,
+                         static_cast<cudaStream_t>(cuda_stream));
 }
 
 int mv_set_cameras(mv_batch *b, const mv_camera *d_cams, void *cuda_stream) {
@@ -538,7 +573,7 @@ int mv_step_host(mv_batch *b, const mv_camera *h_cams, const mv_box *h_boxes, co
         MV_CUDA(b, cudaMemcpyAsync(b->d_box_in, h_boxes, (size_t)E * b->desc.max_boxes * sizeof(mv_box),
                                    cudaMemcpyHostToDevice, s));
         MV_CUDA(b, cudaMemcpyAsync(b->d_count_in, h_box_count, (size_t)E * sizeof(int32_t), cudaMemcpyHostToDevice, s));
-        int r = launch_boxes(b, 0, E, b->d_box_in, b->d_count_in, s);
+        int r = launch_boxes(b, 0, nullptr, E, b->d_box_in, b->d_count_in, s);
         if (r != MV_OK) return r;
     }
     int r = launch_cameras(b, b->d_cam_in, s);
@@ -646,7 +681,7 @@ int mv_destroy(mv_batch *b) {
         if (g.ok) {
             if (cudaDeviceSynchronize() != cudaSuccess) rc = MV_ERR_CUDA;
             cudaFree(b->d_env_blocks); cudaFree(b->d_mat); cudaFree(b->d_cams); cudaFree(b->d_status);
-            cudaFree(b->d_overlay); cudaFree(b->d_overlay_count); cudaFree(b->d_covered);
+            cudaFree(b->d_overlay); cudaFree(b->d_overlay_count); cudaFree(b->d_covered); cudaFree(b->d_env_index);
             free_host_step(b);
             cudaGetLastError();
         }

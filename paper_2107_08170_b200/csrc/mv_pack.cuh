@@ -20,12 +20,17 @@ __device__ __forceinline__ void transpose4x4(const uint32_t in[4], uint32_t out[
     out[2] = __byte_perm(c, d, 0x5410); out[3] = __byte_perm(c, d, 0x7632);
 }
 
+// Destination env of the e-th env of an upload: a contiguous range, or an index list.
+__device__ __forceinline__ size_t upload_env(const int32_t *__restrict__ env_index, int env_begin, size_t e) {
+    return env_index ? (size_t)__ldg(env_index + e) : (size_t)env_begin + e;
+}
+
 // uint8 grid [env][y][z][x] -> occupancy bits packed along y inside the env block (see EnvLayout)
 // plus a material copy by voxel index with ids clamped to the palette.  One thread packs 32
 // heights of four neighbouring columns: 32 four-byte loads, four words and 128 material bytes out.
 __global__ void pack_grid_kernel(const uint8_t *__restrict__ grid, unsigned char *__restrict__ env_blocks,
                                  uint8_t *__restrict__ mat, EnvLayout lay, int gx, int gy, int gz, int env_begin,
-                                 int env_count, int palette, uint32_t *status)
+                                 const int32_t *__restrict__ env_index, int env_count, int palette, uint32_t *status)
 {
     const int xg_n = gx / 4, col_words = 1 << (lay.ysh - 5);
     const size_t per_env = (size_t)xg_n * gz * col_words;
@@ -40,7 +45,7 @@ __global__ void pack_grid_kernel(const uint8_t *__restrict__ grid, unsigned char
     const uint8_t *src = grid + e * nvox + (size_t)z * gx + 4 * xg;
     const uint32_t cap = (uint32_t)(palette - 1) * 0x01010101u;
     uint32_t bits[4] = {0, 0, 0, 0}, clamped = 0;
-    const size_t env = (size_t)env_begin + e;
+    const size_t env = upload_env(env_index, env_begin, e);
     const uint32_t u0 = voxel_index(lay.ysh, gx, 4 * xg, 32 * wq, z);
     uint8_t *mdst = mat + env * ((size_t)gx * gz << lay.ysh) + u0;
     uint32_t col[4][8];                                 // material bytes: column c, heights 4k..4k+3 in word k
@@ -77,9 +82,9 @@ __global__ void pack_grid_kernel(const uint8_t *__restrict__ grid, unsigned char
 // Cell box [lo, hi) that contains every filled voxel of an env, from the packed occupancy bits.
 // One CTA per env; written next to the box count.  An empty grid gives lo > hi.
 __global__ void occupied_bounds_kernel(unsigned char *__restrict__ env_blocks, EnvLayout lay, int env_begin,
-                                       int gx, int gy, int gz)
+                                       const int32_t *__restrict__ env_index, int gx, int gy, int gz)
 {
-    unsigned char *blk = env_blocks + (size_t)(env_begin + blockIdx.x) * lay.stride;
+    unsigned char *blk = env_blocks + upload_env(env_index, env_begin, blockIdx.x) * lay.stride;
     const uint32_t *occ = reinterpret_cast<const uint32_t *>(blk);
     const int wsh = lay.ysh - 5;                   // log2 of the words per column
     const int nwords = (gx * gz) << wsh;
@@ -112,7 +117,7 @@ __global__ void occupied_bounds_kernel(unsigned char *__restrict__ env_blocks, E
 
 // Shaded colour table per env: lut[face][m] = RGBX of floor(palette*I_face + 0.5), in double.
 __global__ void build_lut_kernel(const uint8_t *__restrict__ palette, unsigned char *__restrict__ env_blocks,
-                                 EnvLayout lay, int env_begin, int env_count, int P,
+                                 EnvLayout lay, int env_begin, const int32_t *__restrict__ env_index, int env_count, int P,
                                  double lx, double ly, double lz, double ambient)
 {
     const int gid = blockIdx.x * blockDim.x + threadIdx.x;
@@ -136,20 +141,21 @@ __global__ void build_lut_kernel(const uint8_t *__restrict__ palette, unsigned c
         v = v > 255.0 ? 255.0 : v;
         out |= (uint32_t)v << (8 * c);
     }
-    uint32_t *lut = reinterpret_cast<uint32_t *>(env_blocks + (size_t)(env_begin + e) * lay.stride + lay.lut_off);
+    uint32_t *lut = reinterpret_cast<uint32_t *>(env_blocks + upload_env(env_index, env_begin, e) * lay.stride + lay.lut_off);
     lut[f * P + m] = out;
 }
 
 // Box lists into the env blocks; material ids and counts are clamped.
 __global__ void copy_boxes_kernel(const uint4 *__restrict__ boxes, const int32_t *__restrict__ counts,
                                   unsigned char *__restrict__ env_blocks, EnvLayout lay, int env_begin,
-                                  int env_count, int max_boxes, int palette, uint32_t *status)
+                                  const int32_t *__restrict__ env_index, int env_count, int max_boxes, int palette,
+                                  uint32_t *status)
 {
     const int gid = blockIdx.x * blockDim.x + threadIdx.x;
     const int per_env = max_boxes + 1;
     if (gid >= env_count * per_env) return;
     const int e = gid / per_env, b = gid - e * per_env;
-    unsigned char *blk = env_blocks + (size_t)(env_begin + e) * lay.stride;
+    unsigned char *blk = env_blocks + upload_env(env_index, env_begin, e) * lay.stride;
     if (b == max_boxes) {
         int n = counts[e];
         if (n < 0 || n > max_boxes) { n = n < 0 ? 0 : max_boxes; atomicOr(status, kFlagBoxCount); }

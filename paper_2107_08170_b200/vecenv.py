@@ -9,8 +9,7 @@ tensors owned by this object (Section 3.2: frames exposed directly as GPU-side t
 
 Built for thousands of environments: episode clocks, the time-left rectangles and the agent state
 live on the GPU; per step the host only learns which environments finished (one small read), then
-generates all of their new worlds in one batch and uploads them run by run of neighbouring
-environment indices."""
+generates all of their new worlds in one batch and uploads them with one scattered upload."""
 from __future__ import annotations
 
 import torch
@@ -34,18 +33,6 @@ def time_bar_rects(steps_left, episode_len, width, agents):
     rec[:, 0, 1] = x1.to(torch.int32) | (BAR_ROWS << 16)   # x1 (low half), y1 (high half); x0 = y0 = 0
     rec[:, 0, 2] = BAR_RGB[0] | (BAR_RGB[1] << 8) | (BAR_RGB[2] << 16)
     return rec
-
-
-def _runs(sorted_idx):
-    """[(start position, length)] of the runs of consecutive integers in a sorted list."""
-    out, i, n = [], 0, len(sorted_idx)
-    while i < n:
-        j = i
-        while j + 1 < n and sorted_idx[j + 1] == sorted_idx[j] + 1:
-            j += 1
-        out.append((i, j - i + 1))
-        i = j + 1
-    return out
 
 
 class VecRenderEnv:
@@ -76,12 +63,10 @@ class VecRenderEnv:
             chunk = envs[c0:c0 + _GEN_CHUNK]
             ids = torch.tensor([e + int(ep[e]) * cfg.num_envs for e in chunk], dtype=torch.int64)
             sc = scenes.make_scene(cfg, device=self.device, env_ids=ids)
-            for i0, n in _runs(chunk):
-                boxes = count = None
-                if cfg.max_boxes > 0:
-                    boxes, count = sc["boxes"][i0:i0 + n].contiguous(), sc["box_count"][i0:i0 + n].contiguous()
-                self.batch.upload_worlds(chunk[i0], n, sc["grid"][i0:i0 + n].contiguous(), boxes, count,
-                                         sc["palette"][i0:i0 + n].contiguous())
+            boxes = count = None
+            if cfg.max_boxes > 0:
+                boxes, count = sc["boxes"].contiguous(), sc["box_count"].contiguous()
+            self.batch.upload_worlds_at(chunk, sc["grid"].contiguous(), boxes, count, sc["palette"].contiguous())
             obs = (torch.tensor(chunk, device=self.device)[:, None] * A + torch.arange(A, device=self.device)).flatten()
             self.cams[obs] = sc["cams"]
 

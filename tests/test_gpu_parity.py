@@ -306,6 +306,55 @@ def test_not_ready_and_argument_errors():
     batch.destroy()
 
 
+def test_scattered_upload_equals_env_by_env_upload():
+    """mv_upload_worlds_at writes env i of its arrays to the listed env: the same bytes as one
+    contiguous upload per listed env; readiness is tracked per listed env; bad lists are refused."""
+    from gpu_util import upload_scene
+    B = _binding()
+    cfg = scenes.config("rooms_boxes", num_envs=12)
+    old, new = scenes.make_scene(cfg), scenes.make_scene(scenes.config("rooms_boxes", num_envs=12, seed=91))
+    where = [1, 4, 5, 9]
+    dev = lambda t: t.cuda().contiguous()
+    frames = []
+    for scattered in (False, True):
+        batch = B.Batch(B.desc_from_config(cfg))
+        upload_scene(batch, old)
+        if scattered:
+            batch.upload_worlds_at(where, dev(new["grid"][:4]), dev(new["boxes"][:4]), dev(new["box_count"][:4]),
+                                   dev(new["palette"][:4]))
+        else:
+            for i, e in enumerate(where):
+                batch.upload_worlds(e, 1, dev(new["grid"][i:i + 1]), dev(new["boxes"][i:i + 1]),
+                                    dev(new["box_count"][i:i + 1]), dev(new["palette"][i:i + 1]))
+        batch.set_cameras(old["cams"].cuda())
+        rgb, depth = batch.alloc_outputs()
+        batch.render_batch(rgb, depth)
+        assert batch.query_status() == 0
+        frames.append((rgb.cpu(), depth.cpu()))
+        batch.destroy()
+    assert torch.equal(frames[0][0], frames[1][0]) and torch.equal(frames[0][1], frames[1][1])
+    A = cfg.agents
+    changed = [bool((frames[1][0][e * A:(e + 1) * A] != 0).any()) for e in range(12)]
+    assert all(changed)
+    # readiness: only the listed envs count as uploaded
+    batch = B.Batch(B.desc_from_config(cfg))
+    batch.upload_worlds_at([0, 2, 11], dev(new["grid"][:3]), None, None, dev(new["palette"][:3]))
+    batch.set_cameras(old["cams"].cuda())
+    rgb, depth = batch.alloc_outputs()
+    with pytest.raises(B.MvError) as ei:
+        batch.render_batch(rgb, depth)
+    assert ei.value.code == -4
+    rest = [e for e in range(12) if e not in (0, 2, 11)]
+    batch.upload_worlds_at(rest, dev(old["grid"][:9]), None, None, dev(old["palette"][:9]))
+    batch.render_batch(rgb, depth)
+    for bad in ([3, 3], [5, 4], [-1, 2], [0, 12]):
+        with pytest.raises(B.MvError) as ei:
+            batch.upload_worlds_at(bad, dev(new["grid"][:2]), None, None, dev(new["palette"][:2]))
+        assert ei.value.code == -1
+    batch.upload_worlds_at([], None, None, None, None)          # nothing to do
+    batch.destroy()
+
+
 def test_limits_are_reported_not_faulted():
     B = _binding()
     import ctypes as C
