@@ -21,11 +21,13 @@ namespace {
 #endif
 constexpr int kRenderThreads = MV_NT;
 constexpr int kHostChunks = 8;
-// Staging + set-up of a CTA, in units of one observation's render time, as measured: 0.13 to 0.19 for
-// 128x72 images of small grids (four or more CTAs per SM); nothing measurable for grids whose block
-// leaves room for three CTAs per SM, where longer CTAs only make the last wave coarser.
+// Staging + set-up of a CTA, in units of one observation's render time, as measured on B200: 0.15 to
+// 0.18 for 128x72 images of 64x16x64 grids (16 KB of occupancy per env); nothing measurable for
+// 128x32x128 grids (64 KB), where sharing a staged block among agents only makes the CTAs longer and the
+// last wave coarser.
 constexpr double kCtaFixedCost = 0.15;
 constexpr double kCtaFixedCostBigBlock = 0.0;
+constexpr uint32_t kBigBlockBytes = 32u << 10;
 constexpr size_t kMergeScratchBytes = 256u << 20;   // coverage bitmap for the envs of one merge launch
 
 inline uint32_t round_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
@@ -420,7 +422,7 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
                                                                               m.bytes - unstaged);
                 if (q != cudaSuccess || per_sm < 1) return 1e30;
                 const double slots = (double)per_sm * sms, ctas = (double)b->num_obs / apc;
-                return std::ceil(ctas / slots) * (apc + (per_sm >= 4 ? kCtaFixedCost : kCtaFixedCostBigBlock));
+                return std::ceil(ctas / slots) * (apc + (L.block_bytes <= kBigBlockBytes ? kCtaFixedCost : kCtaFixedCostBigBlock));
             };
             if (waves_cost(all, d.agents_per_env) < waves_cost(b->smem, 1)) {
                 b->smem = all;

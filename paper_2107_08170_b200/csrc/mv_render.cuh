@@ -546,7 +546,13 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             // per environment) and the GUI overlay.  A box wins only with a strictly smaller time.
             if ((m | rare) != 0u) {
                 if (p.max_boxes < 32) m &= ~kOverlayTileBit;
-                if (m != 0u || mw > 1) {
+                uint32_t any_box = m;
+                for (int w = 1; w < mw; ++w) {       // (more than 32 boxes per env: the tile's other mask words)
+                    uint32_t mm;
+                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(mm) : "r"(mask_p + 4u * (uint32_t)w));
+                    any_box |= mm;
+                }
+                if (any_box != 0u) {
                     // signed reciprocals again, and the ray's rows of the DDA table for the faces
                     const float ix = __uint_as_float(__float_as_uint(dtx) | (sgn3 << 31));
                     const float iy = __uint_as_float(__float_as_uint(dty) | ((sgn3 & 2u) << 30));

@@ -222,7 +222,11 @@ def _world_rooms(rng: Rng, env, gx, gy, gz, P, n_lines=6, pitch=9, n_pillars=24)
     px = rng.randint(28, e1, pi, 1, gx - 2)
     pz = rng.randint(29, e1, pi, 1, gz - 2)
     pm = rng.randint(30, e1, pi, 1, P - 1)
-    M2 = M2.reshape(E, -1).scatter(1, pz * gx + px, pm).reshape(E, gz, gx)
+    # two pillars can fall on one cell: the one with the higher index wins (a maximum over keys, which has
+    # one result on every device; a plain scatter with repeated indices does not)
+    won = torch.zeros(E, gz * gx, dtype=torch.int64, device=dev)
+    won.scatter_reduce_(1, pz * gx + px, pi * 256 + pm, reduce="amax", include_self=True)
+    M2 = torch.where(won > 0, won & 255, M2.reshape(E, -1)).reshape(E, gz, gx)
     height = torch.where(M2 > 0, gy - 1, 0)
     return height, M2, floor
 

@@ -236,3 +236,16 @@ def test_tall_grid_with_multi_word_columns(oracle):
         assert (after[o] == new).all(), (o, after[o], new)
     assert after[0, 2] == 2.0 and after[1, 2] == 4.0          # blocked by the block at z = 3 up there, free below it
     batch.destroy()
+
+
+def test_scene_generators_give_the_same_arrays_on_cpu_and_gpu():
+    """Seeded inputs must not depend on the device or on the order in which a device applies writes
+    (two pillars of a rooms world can fall on the same cell): 1024 envs generated on the GPU twice and
+    on the CPU once are the same arrays."""
+    for name in ("rooms_boxes", "headline"):
+        cfg = scenes.config(name, num_envs=1024 if name == "rooms_boxes" else 64)
+        cpu = scenes.make_scene(cfg)
+        for _ in range(2):
+            gpu = scenes.make_scene(cfg, device=torch.device("cuda", 0))
+            for k in ("grid", "palette", "boxes", "box_count", "cams"):
+                assert torch.equal(cpu[k], gpu[k].cpu()), (name, k)
