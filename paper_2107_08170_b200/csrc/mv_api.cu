@@ -116,7 +116,9 @@ mv_batch::Smem smem_layout(const mv_batch *b, int apc) {
     m.agent_off = m.tile_off + ntiles * 16;
     m.agent_ov_off = kAgentRelOff + (uint32_t)(d.max_boxes > 0 ? d.max_boxes : 1) * 32;
     m.agent_mask_off = m.agent_ov_off + (uint32_t)(d.max_overlay_rects > 0 ? d.max_overlay_rects : 1) * 32;
-    m.agent_ovtile_off = m.agent_mask_off + round_up(ntiles * (uint32_t)b->mask_words * 4, 16);
+    // per tile: the box-mask words, preceded by a summary word when there is more than one
+    const uint32_t words_per_tile = b->mask_words > 1 ? (uint32_t)b->mask_words + 1 : 1u;
+    m.agent_ovtile_off = m.agent_mask_off + round_up(ntiles * words_per_tile * 4, 16);
     m.agent_stride = m.agent_ovtile_off + round_up(((ntiles + 31) / 32) * 4, 16);
     m.misc_off = m.agent_off + (uint32_t)apc * m.agent_stride;
     m.bytes = m.misc_off + 32;

@@ -217,7 +217,11 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     const int env = obs0 / p.agents;
     const int W = p.W, H = p.H;
     const int ntiles = p.tiles_x * p.tiles_y;
+    // Box masks per tile: mw words of one bit per box.  With more than 32 boxes a summary word (the OR of
+    // the others) comes first, so that the per-tile test reads one word whatever the box count.
     const int mw = p.mask_words;
+    const int ms = mw > 1 ? mw + 1 : 1;              // words per tile
+    const int m0 = mw > 1 ? 1 : 0;                   // position of the first real mask word
 
     // bytes of the env block that are NOT staged (the occupancy, when it stays in global memory)
     const uint32_t unstaged = OCC_SHARED ? 0u : p.lay.occ_bytes;
@@ -249,7 +253,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     // ---- meanwhile: tile table, cleared masks, camera records, GUI rectangles
     for (int ag = 0; ag < apc; ++ag) {
         uint32_t *mk = agent_mask(ag);
-        for (int i = tid; i < ntiles * mw; i += NT) mk[i] = 0u;
+        for (int i = tid; i < ntiles * ms; i += NT) mk[i] = 0u;
     }
     const float inv_tiles_x = 1.0f / (float)p.tiles_x;
     for (int i = tid; i < ntiles; i += NT) {
@@ -419,7 +423,11 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             uint32_t *mask = agent_mask(ag);
             for (int ty = py0 >> 2; ty <= (py1 >> 2); ++ty)
                 for (int tx = px0 >> 3; tx <= (px1 >> 3); ++tx)
-                    atomicOr(&mask[(ty * p.tiles_x + tx) * mw + (b >> 5)], bit);
+                    {
+                        uint32_t *tm = mask + (ty * p.tiles_x + tx) * ms;
+                        atomicOr(tm + m0 + (b >> 5), bit);
+                        if (mw > 1) atomicOr(tm, bit);          // the summary word only has to be non-zero
+                    }
         }
     }
 #if MV_BRICKS == 1
@@ -463,7 +471,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
 #else
     uint32_t tile_end = smem_addr(s_tile) + 16u * (uint32_t)ntiles;
 #endif
-    uint32_t mask_step = 4u * kWarps * (uint32_t)mw;                        // bytes between a warp's consecutive tile masks
+    uint32_t mask_step = 4u * kWarps * (uint32_t)ms;                        // bytes between a warp's consecutive tile masks
     keep(tile_end); keep(mask_step);
 
     for (int ag = 0; ag < apc; ++ag) {
@@ -479,12 +487,11 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         const float Px = c0.x, Py = c0.y, Pz = c0.z;
         const bool cam_in = (aflags & kAgentInside) != 0;
         const int ov_count = __float_as_int(c3.w);
-        // non-zero: every tile takes the slow branch (more than one mask word per tile, or an overlay that
-        // cannot flag its tiles in the box mask)
-        uint32_t rare = (mw > 1 ? 1u : 0u) | ((ov_count > 0 && p.max_boxes >= 32) ? 2u : 0u);
+        // non-zero: every tile takes the slow branch (an overlay that cannot flag its tiles in the box mask)
+        uint32_t rare = (ov_count > 0 && p.max_boxes >= 32) ? 2u : 0u;
         keep(rare);
         uint32_t abase = smem_addr(agent_rec(ag));
-        uint32_t mask_p = smem_addr(agent_mask(ag) + (size_t)warp * mw);
+        uint32_t mask_p = smem_addr(agent_mask(ag) + (size_t)warp * ms);
         // (store addresses as global-space addresses for the PTX store block)
         unsigned long long depth_lane = (unsigned long long)__cvta_generic_to_global(depth_obs + depth_lane_off);
         unsigned long long rgb_lane = (unsigned long long)__cvta_generic_to_global(rgb_obs + rgb_lane_off);
@@ -546,13 +553,9 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
             // per environment) and the GUI overlay.  A box wins only with a strictly smaller time.
             if ((m | rare) != 0u) {
                 if (p.max_boxes < 32) m &= ~kOverlayTileBit;
-                uint32_t any_box = m;
-                for (int w = 1; w < mw; ++w) {       // (more than 32 boxes per env: the tile's other mask words)
-                    uint32_t mm;
-                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(mm) : "r"(mask_p + 4u * (uint32_t)w));
-                    any_box |= mm;
-                }
-                if (any_box != 0u) {
+                if (m != 0u) {
+                    // (more than 32 boxes per env: m was the summary; start with the first real word)
+                    if (mw > 1) asm volatile("ld.shared.u32 %0, [%1+4];" : "=r"(m) : "r"(mask_p));
                     // signed reciprocals again, and the ray's rows of the DDA table for the faces
                     const float ix = __uint_as_float(__float_as_uint(dtx) | (sgn3 << 31));
                     const float iy = __uint_as_float(__float_as_uint(dty) | ((sgn3 & 2u) << 30));
@@ -584,7 +587,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                             }
                         }
                         if (++w >= mw) break;
-                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(m) : "r"(mask_p + 4u * (uint32_t)w));
+                        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(m) : "r"(mask_p + 4u * (uint32_t)(w + m0)));
                     }
                     if (baddr) {
                         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(rgbx) : "r"(baddr));
