@@ -504,12 +504,13 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         // lanes, so they wait by themselves for lanes whose walk ran longer.
         auto finish_tile = [&](uint32_t tile_p, uint32_t mask_p, int tile_px, uint32_t pos, uint32_t bit, uint32_t row,
                                uint32_t sgn3, float t_hit, float dtx, float dty, float dtz) {
-            // ---- voxel colour (one material byte from global memory, then the shaded table), this
-            // tile's first box-mask word, and the latest voxel hit of the warp (boxes wholly behind it
-            // are skipped).  Predicated, not branched; sky colour and miss depth ride with the material
-            // store's address in the agent block.  (Column-word flavour: the voxel index is rebuilt from
+            // ---- the hit voxel's material byte is asked for from global memory (its colour is looked up
+            // in the shaded table only in the store block, after everything that does not need it), this
+            // tile's first box-mask word is read, and the latest voxel hit of the warp is found (boxes wholly
+            // behind it are skipped).  Predicated, not branched; sky colour and miss depth ride with the
+            // material store's address in the agent block.  (Column-word flavour: the voxel index is rebuilt from
             // the column's address and the bit.)
-            uint32_t rgbx, m;
+            uint32_t rgbx, m, mat_id;
             float depth, tb, wmax;
             {
                 uint32_t vi = pos;
@@ -520,25 +521,23 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                 }
                 asm volatile("{\n"
                     " .reg .pred pv;\n"
-                    " .reg .b32 mid, skyb, missb, tbb, wmb;\n"
+                    " .reg .b32 skyb, missb, tbb, wmb;\n"
                     " .reg .b64 mp, sm;\n"
-                    " ld.shared.v2.b64 {mp, sm}, [%8+80];\n"
-                    " ld.shared.u32 %2, [%9];\n"
+                    " ld.shared.v2.b64 {mp, sm}, [%9+80];\n"
+                    " ld.shared.u32 %2, [%10];\n"
                     " mov.b64 {skyb, missb}, sm;\n"
                     " mov.b32 %0, skyb;\n"
                     " mov.b32 %1, missb;\n"
-                    " setp.ne.u32 pv, %5, 0xffffffff;\n"
-                    " mad.wide.u32 mp, %6, 1, mp;\n"
-                    " mov.b32 tbb, %7;\n"
-                    " @pv ld.global.nc.u8 mid, [mp];\n"
-                    " @pv mad.lo.u32 mid, mid, 4, %5;\n"
+                    " setp.ne.u32 pv, %6, 0xffffffff;\n"
+                    " mad.wide.u32 mp, %7, 1, mp;\n"
+                    " mov.b32 tbb, %8;\n"
+                    " @pv ld.global.nc.u8 %5, [mp];\n"
                     " redux.sync.max.u32 wmb, tbb, 0xffffffff;\n"
                     " mov.b32 %3, tbb;\n"
                     " mov.b32 %4, wmb;\n"
-                    " @pv ld.shared.u32 %0, [mid];\n"
-                    " @pv mov.f32 %1, %7;\n"
+                    " @pv mov.f32 %1, %8;\n"
                     "}\n"
-                    : "=&r"(rgbx), "=&f"(depth), "=&r"(m), "=&f"(tb), "=&f"(wmax)
+                    : "=&r"(rgbx), "=&f"(depth), "=&r"(m), "=&f"(tb), "=&f"(wmax), "=&r"(mat_id)
                     : "r"(row), "r"(vi), "f"(t_hit), "r"(abase), "r"(mask_p)
                     : "memory");
             }
@@ -592,6 +591,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                     if (baddr) {
                         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(rgbx) : "r"(baddr));
                         depth = tb + 0.0f;
+                        row = kNoRow;                            // the voxel behind the box is not looked up
                     }
                 }
                 // GUI overlay: rectangles in list order, later ones on top; depth is left alone
@@ -600,6 +600,10 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
                     if ((agent_ovtile(ag)[tile_no >> 5] >> (tile_no & 31)) & 1u) {
                         const int4 *ov = agent_ov(ag);
                         const int px = (tile_px % W) + (lane & 7), py = (tile_px / W) + (lane >> 3);
+                        if (row != kNoRow) {                     // the rectangles go over the voxel colour: look it up now
+                            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(rgbx) : "r"(row + 4u * mat_id));
+                            row = kNoRow;
+                        }
                         for (int r = 0; r < ov_count; ++r) {
                             const int4 q = ov[2 * r];
                             if (px >= q.x && px < q.z && py >= q.y && py < q.w) rgbx = (uint32_t)ov[2 * r + 1].x;
@@ -610,18 +614,22 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
 
             // ---- store: depth rows are 32-byte segments; RGB rows are 24 bytes = 6 packed words
             asm volatile("{\n"
-                " .reg .pred ps;\n"
-                " .reg .b32 ca, cb;\n"
+                " .reg .pred ps, pv;\n"
+                " .reg .b32 ca, cb, cc;\n"
                 " .reg .b64 ad;\n"
                 " mad.wide.s32 ad, %2, 4, %3;\n"
                 " st.global.f32 [ad], %1;\n"
-                " shfl.sync.down.b32 cb, %0, 1, 31, 0xffffffff;\n"
+                " setp.ne.u32 pv, %6, 0xffffffff;\n"
+                " mad.lo.u32 ca, %7, 4, %6;\n"
+                " mov.b32 cc, %0;\n"
+                " @pv ld.shared.u32 cc, [ca];\n"
+                " shfl.sync.down.b32 cb, cc, 1, 31, 0xffffffff;\n"
                 " mad.wide.s32 ad, %2, 3, %4;\n"
-                " prmt.b32 ca, %0, cb, %5;\n"
+                " prmt.b32 ca, cc, cb, %5;\n"
                 " setp.ge.s32 ps, %5, 0;\n"
                 " @ps st.global.u32 [ad], ca;\n"
                 "}\n"
-                :: "r"(rgbx), "f"(depth), "r"(tile_px), "l"(depth_lane), "l"(rgb_lane), "r"(st_sel)
+                :: "r"(rgbx), "f"(depth), "r"(tile_px), "l"(depth_lane), "l"(rgb_lane), "r"(st_sel), "r"(row), "r"(mat_id)
                 : "memory");
         };
         if (COLW && cam_in && !MV_BRICKS) {
