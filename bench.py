@@ -75,18 +75,25 @@ class ClockSampler:
             self._err = repr(e)
             self._h = None
 
-    def _run(self):
+    def sample_now(self):
+        """One sample from the calling thread (the timed loop calls it while its launches are still
+        running on the GPU, so a short timed region has a sample under load even if the thread got no turn)."""
+        if self._h is None:
+            return
         nv = self._nv
+        try:
+            self.samples.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+            r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+            for bit, name in ((self.HW_SLOWDOWN, "hw_slowdown"), (self.HW_THERMAL, "hw_thermal_slowdown"),
+                              (self.SW_THERMAL, "sw_thermal_slowdown"), (self.SW_POWER, "sw_power_cap")):
+                if r & bit:
+                    self.reasons.add(name)
+        except Exception:               # noqa: BLE001
+            pass
+
+    def _run(self):
         while not self._stop.is_set():
-            try:
-                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
-                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
-                for bit, name in ((self.HW_SLOWDOWN, "hw_slowdown"), (self.HW_THERMAL, "hw_thermal_slowdown"),
-                                  (self.SW_THERMAL, "sw_thermal_slowdown"), (self.SW_POWER, "sw_power_cap")):
-                    if r & bit:
-                        self.reasons.add(name)
-            except Exception:           # noqa: BLE001
-                pass
+            self.sample_now()
             self._stop.wait(0.002)
 
     def start(self):
@@ -381,6 +388,7 @@ def main():
         batch.render_batch(rgb, depth)
         e2.record(stream)
     t_end.record(stream)
+    sampler.sample_now()                       # the launches above are still running
     barrier()
     total_ms = t_begin.elapsed_time(t_end)
     if flush is not None:                      # the flushes sit between the steps: sum the steps alone
