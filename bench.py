@@ -189,7 +189,7 @@ def time_extras(batch, cfg, cams, rgb, depth, dev):
     moves = ((torch.rand(cfg.num_obs, 4, device=dev) - 0.5) * torch.tensor([0.4, 0.2, 0.3, 0.1], device=dev)).contiguous()
     out["move_agents_ms"] = med(lambda: batch.move_agents(moved, moves))
     out["set_cameras_ms"] = med(lambda: batch.set_cameras(cams))
-    n = min(E, 2048)
+    n = min(E, 8192)
     out["merge_voxels_ms_per_env"] = med(lambda: batch.merge_voxels(0, n, 2048), 3) / n
     out["merged_boxes_per_env"] = float(batch.merge_voxels(0, n, 2048)[1].float().mean())
     batch.debug_occupancy_in_global(True)

@@ -188,7 +188,7 @@ int mv_render_batch(mv_batch *batch, uint8_t *d_rgb, float *d_depth, void *cuda_
  *   d_boxes_out DEVICE mv_box [env_count][max_out]; box b of an env is valid for b < min(count, max_out)
  *   d_count_out DEVICE int32 [env_count]; the number of boxes the sweep produces (may exceed max_out,
  *               in which case only the first max_out were written)
- * The first call allocates scratch (2 bits per voxel for as many envs as fit in 256 MiB: the
+ * The first call allocates scratch (2 bits per voxel for as many envs as fit in 1 GiB, at most the batch: the
  * coverage bitmap and a copy of the occupancy in sweep order).
  * Errors: INVALID_ARG, NOT_READY (an env in the range has no grid), OUT_OF_MEMORY, CUDA. */
 int mv_merge_voxels(mv_batch *batch, int env_begin, int env_count, mv_box *d_boxes_out,

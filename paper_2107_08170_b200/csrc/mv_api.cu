@@ -28,7 +28,10 @@ constexpr int kHostChunks = 8;
 constexpr double kCtaFixedCost = 0.15;
 constexpr double kCtaFixedCostBigBlock = 0.0;
 constexpr uint32_t kBigBlockBytes = 32u << 10;
-constexpr size_t kMergeScratchBytes = 256u << 20;   // coverage bitmap for the envs of one merge launch
+#ifndef MV_MERGE_SCRATCH_MB
+#define MV_MERGE_SCRATCH_MB 1024
+#endif
+constexpr size_t kMergeScratchBytes = (size_t)MV_MERGE_SCRATCH_MB << 20;   // coverage bitmap for the envs of one merge launch
 
 inline uint32_t round_up(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
 

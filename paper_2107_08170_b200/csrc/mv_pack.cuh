@@ -344,12 +344,27 @@ __global__ void merge_voxels_kernel(const uint32_t *__restrict__ occx, const uin
                 if (!__all_sync(full, ok)) break;
             }
             __syncwarp();
-            for (int c = lane; c < w * d * h; c += 32) {         // mark covered
-                const int a = c % w, b = (c / w) % d, cc = c / (w * d);
-                const int vv = (i + a) + gx * ((k + b) + gz * (j + cc));
-                atomicOr(&cov[vv >> 5], 1u << (vv & 31));
+            // mark covered.  When gx is a multiple of 32, x-rows of different z or y never share a word:
+            // one lane per row does plain read-modify-writes, and the warp barrier orders them before the
+            // other lanes' later reads.  Narrower grids take atomics and a fence.
+            if ((gx & 31) == 0) {
+                for (int r = lane; r < d * h; r += 32) {
+                    const int b = r % d, cc = r / d;
+                    const int v0 = i + gx * ((k + b) + gz * (j + cc)), v1 = v0 + w;      // bits [v0, v1)
+                    for (int wd = v0 >> 5; wd <= (v1 - 1) >> 5; ++wd) {
+                        const int lo = max(v0 - 32 * wd, 0), hi = min(v1 - 32 * wd, 32);
+                        const uint32_t bits = (hi == 32 ? 0xffffffffu : ((1u << hi) - 1u)) & ~((1u << lo) - 1u);
+                        __stcg(&cov[wd], __ldcg(&cov[wd]) | bits);
+                    }
+                }
+            } else {
+                for (int c = lane; c < w * d * h; c += 32) {
+                    const int a = c % w, b = (c / w) % d, cc = c / (w * d);
+                    const int vv = (i + a) + gx * ((k + b) + gz * (j + cc));
+                    atomicOr(&cov[vv >> 5], 1u << (vv & 31));
+                }
+                __threadfence();
             }
-            __threadfence();                                     // marks visible to the other lanes' reads
             __syncwarp();
             if (lane == 0 && count < max_out) {
                 out[2 * count] = make_uint4(__float_as_uint((float)i), __float_as_uint((float)j),
