@@ -8,8 +8,9 @@ time-left bar of Appendix A.2 is drawn through the GUI overlay.  Observations ar
 tensors owned by this object (Section 3.2: frames exposed directly as GPU-side tensors).
 
 Built for thousands of environments: episode clocks, the time-left rectangles and the agent state
-live on the GPU; per step the host only learns which environments finished (one small read), then
-generates all of their new worlds in one batch and uploads them with one scattered upload."""
+live on the GPU; per step the host only learns which environments finished (one small read) and
+uploads their new worlds with one scattered upload.  Episode lengths are fixed, so the worlds that
+the next few steps will need are known in advance and are generated together, a window at a time."""
 from __future__ import annotations
 
 import torch
@@ -19,6 +20,7 @@ from . import binding, scenes
 BAR_RGB = (250, 240, 30)
 BAR_ROWS = 2
 _GEN_CHUNK = 512            # environments generated per scene-generator call
+_LOOKAHEAD = 8              # steps whose resets are generated together
 
 
 def time_bar_rects(steps_left, episode_len, width, agents):
@@ -52,23 +54,65 @@ class VecRenderEnv:
         self.episode = torch.zeros(E, dtype=torch.int64, device=self.device)
         self._bar_count = torch.ones(cfg.num_obs, dtype=torch.int32, device=self.device)
         self._started = False
+        self._step = 0                      # steps taken so far
+        self._ahead = {}                    # step number -> (env list, their generated scenes) for coming resets
 
-    def _load_envs(self, envs):
-        """Fresh worlds for the (sorted) local env indices in `envs`; env e in its k-th episode uses the
-        seeded scene id e + k * num_envs."""
-        cfg, A = self.cfg, self.cfg.agents
-        envs = [int(e) for e in envs]
-        ep = self.episode.cpu()
+    def _generate(self, envs, episodes):
+        """Scenes (a list of chunks) for the env indices `envs` in the given episodes: env e in its k-th
+        episode uses the seeded scene id e + k * num_envs."""
+        out = []
         for c0 in range(0, len(envs), _GEN_CHUNK):
             chunk = envs[c0:c0 + _GEN_CHUNK]
-            ids = torch.tensor([e + int(ep[e]) * cfg.num_envs for e in chunk], dtype=torch.int64)
-            sc = scenes.make_scene(cfg, device=self.device, env_ids=ids)
+            ids = torch.tensor([e + k * self.cfg.num_envs for e, k in zip(chunk, episodes[c0:c0 + _GEN_CHUNK])],
+                               dtype=torch.int64)
+            out.append((chunk, scenes.make_scene(self.cfg, device=self.device, env_ids=ids)))
+        return out
+
+    def _install(self, chunks, pick=None):
+        """Upload generated scenes; `pick` (env list, position range) takes a slice of a single chunk."""
+        A = self.cfg.agents
+        for chunk, sc in chunks:
+            lo, hi = (0, len(chunk)) if pick is None else pick
+            envs = chunk[lo:hi]
+            if not envs:
+                continue
             boxes = count = None
-            if cfg.max_boxes > 0:
-                boxes, count = sc["boxes"].contiguous(), sc["box_count"].contiguous()
-            self.batch.upload_worlds_at(chunk, sc["grid"].contiguous(), boxes, count, sc["palette"].contiguous())
-            obs = (torch.tensor(chunk, device=self.device)[:, None] * A + torch.arange(A, device=self.device)).flatten()
-            self.cams[obs] = sc["cams"]
+            if self.cfg.max_boxes > 0:
+                boxes, count = sc["boxes"][lo:hi].contiguous(), sc["box_count"][lo:hi].contiguous()
+            self.batch.upload_worlds_at(envs, sc["grid"][lo:hi].contiguous(), boxes, count,
+                                        sc["palette"][lo:hi].contiguous())
+            obs = (torch.tensor(envs, device=self.device)[:, None] * A + torch.arange(A, device=self.device)).flatten()
+            self.cams[obs] = sc["cams"][lo * A:hi * A]
+
+    def _load_envs(self, envs):
+        """Fresh worlds for the (sorted) env indices in `envs`, each in its current episode."""
+        envs = [int(e) for e in envs]
+        ep = self.episode.cpu()
+        self._install(self._generate(envs, [int(ep[e]) for e in envs]))
+
+    def _look_ahead(self):
+        """Generate, in one go, the worlds of every env whose episode ends within the next _LOOKAHEAD
+        steps (an env's clock and episode length say when), and file them by the step that needs them."""
+        left = (self.episode_len - self.t).cpu()                # steps until each env finishes (>= 1)
+        ep = self.episode.cpu()
+        horizon = min(_LOOKAHEAD, int(self.episode_len.min()))  # no env finishes twice inside the window
+        when = [(int(left[e]), e) for e in torch.nonzero(left <= horizon).flatten().tolist()]
+        when.sort()
+        envs = [e for _, e in when]
+        chunks = self._generate(envs, [int(ep[e]) + 1 for e in envs])
+        pos = 0
+        for k in range(1, horizon + 1):
+            n = sum(1 for w, _ in when if w == k)
+            mine = envs[pos:pos + n]
+            # the slices of the generated chunks that hold these envs
+            parts, p = [], pos
+            while p < pos + n:
+                ci, off = divmod(p, _GEN_CHUNK)
+                take = min(pos + n - p, _GEN_CHUNK - off)
+                parts.append((chunks[ci], (off, off + take)))
+                p += take
+            self._ahead[self._step + k] = (mine, parts)
+            pos += n
 
     def _render(self):
         if self.time_bar:
@@ -90,13 +134,21 @@ class VecRenderEnv:
         the frames already show the first view of its next episode."""
         assert self._started, "call reset() once before step()"
         self.batch.move_agents(self.cams, moves.contiguous())
+        if not self._ahead:
+            self._look_ahead()
+        self._step += 1
         self.t += 1
         done = self.t >= self.episode_len
         finished = torch.nonzero(done).flatten().cpu().tolist()       # the one device->host read of a step
+        planned = self._ahead.pop(self._step, None)
         if finished:
             self.episode[done] += 1
             self.t[done] = 0
-            self._load_envs(finished)
+            if planned is not None and planned[0] == finished:
+                for chunk, pick in planned[1]:
+                    self._install([chunk], pick)
+            else:
+                self._load_envs(finished)
             self.batch.set_cameras(self.cams)
         rgb, depth = self._render()
         return rgb, depth, done
