@@ -21,13 +21,10 @@ namespace {
 #endif
 constexpr int kRenderThreads = MV_NT;
 constexpr int kHostChunks = 8;
-// Staging + set-up of a CTA, in units of one observation's render time, as measured on B200: 0.15 to
-// 0.18 for 128x72 images of 64x16x64 grids (16 KB of occupancy per env); nothing measurable for
-// 128x32x128 grids (64 KB), where sharing a staged block among agents only makes the CTAs longer and the
-// last wave coarser.
+// Staging + set-up of a CTA, in units of one observation's render time, as measured on B200 at 128x72:
+// 0.15 to 0.18 for 64x16x64 grids, 0.10 for 128x32x128 grids (where a second agent's tables usually cost
+// the third resident CTA per SM, which the occupancy query below sees).
 constexpr double kCtaFixedCost = 0.15;
-constexpr double kCtaFixedCostBigBlock = 0.0;
-constexpr uint32_t kBigBlockBytes = 32u << 10;
 #ifndef MV_MERGE_SCRATCH_MB
 #define MV_MERGE_SCRATCH_MB 1024
 #endif
@@ -427,7 +424,7 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
                                                                               m.bytes - unstaged);
                 if (q != cudaSuccess || per_sm < 1) return 1e30;
                 const double slots = (double)per_sm * sms, ctas = (double)b->num_obs / apc;
-                return std::ceil(ctas / slots) * (apc + (L.block_bytes <= kBigBlockBytes ? kCtaFixedCost : kCtaFixedCostBigBlock));
+                return std::ceil(ctas / slots) * (apc + kCtaFixedCost);
             };
             if (waves_cost(all, d.agents_per_env) < waves_cost(b->smem, 1)) {
                 b->smem = all;
