@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int apc = p.agents_per_cta;
     const int obs0 = p.obs_begin + blockIdx.x * apc;
-    const int env = obs0 / p.agents;
+    const int env = p.agents == 1 ? obs0 : obs0 / p.agents;
     const int W = p.W, H = p.H;
     const int ntiles = p.tiles_x * p.tiles_y;
     // Box masks per tile: mw words of one bit per box.  With more than 32 boxes a summary word (the OR of
@@ -314,7 +314,7 @@ __global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams 
         if (warp == 0 && !p.skip_staging) mbar_wait_bounded(s_bar, 0, kDrainPolls);
         return;
     }
-    mbar_wait_bounded(s_bar, 0, 8);       // completed phase: makes the staged bytes visible to this thread
+    mbar_try_wait(s_bar, 0);              // completed phase: makes the staged bytes visible to this thread
 
     // ---- per-agent traversal set-up and box binning
     const int gx = p.gx, gz = p.gz;
