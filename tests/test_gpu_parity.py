@@ -39,7 +39,10 @@ def _render_custom(oracle, grid, palette, cams, W, H, boxes=None, box_count=None
     batch.destroy()
     if not check:
         return g_rgb, g_depth, status
-    od = oracle.make_desc((gy, gz, gx), max_boxes, W, H, P, **desc_kw)
+    okw = dict(desc_kw)
+    if "hfov_rad" in okw:
+        okw["hfov"] = okw.pop("hfov_rad")                 # the two descriptors name the field differently
+    od = oracle.make_desc((gy, gz, gx), max_boxes, W, H, P, **okw)
     total = None
     for o in range(E * agents):
         e = o // agents
@@ -409,6 +412,53 @@ def test_odd_grid_sizes_and_occupied_bounds(oracle):
         g_rgb, g_depth, status, st = _render_custom(oracle, grid, _pal(2, 4), cams, 64, 36)
         parity.assert_parity(st, f"gx={gx}")
         assert (g_depth[1] == 0).all() and (g_depth[0] > 0).mean() > 0.2
+
+
+@pytest.mark.parametrize("case", [
+    dict(W=8, H=4, grid=(12, 4, 28), P=1, kw=dict(hfov_rad=0.6, ambient=0.0, light_dir=(0.0, 1.0, 0.0))),
+    dict(W=24, H=20, grid=(20, 8, 12), P=256, kw=dict(hfov_rad=2.6, ambient=1.0, miss_depth=-1.0, sky_rgb=(0, 255, 3))),
+    dict(W=136, H=68, grid=(16, 32, 16), P=7, kw=dict(hfov_rad=1.2, light_dir=(-1.0, -0.2, 0.0), miss_depth=1000.0)),
+    dict(W=64, H=36, grid=(36, 12, 8), P=16, kw=dict(light_dir=(0.0, 0.0, -3.0), ambient=0.5)),
+])
+def test_descriptor_corners(oracle, case):
+    """Descriptor fields away from the workloads' defaults: smallest image, image sizes that are no
+    powers of two, narrow and very wide fields of view, one-entry and 256-entry palettes, lights along
+    an axis and from below, ambient 0 and 1, other sky colours and miss depths, flat and full-height grids;
+    boxes and cameras inside and outside the grid."""
+    gx, gy, gz = case["grid"]
+    W, H, P = case["W"], case["H"], case["P"]
+    rng = np.random.default_rng(gx * 1000 + W)
+    E, A, nb = 3, 2, 5
+    if P > 1:
+        grid = ((rng.random((E, gy, gz, gx)) < 0.12) * rng.integers(1, P, size=(E, gy, gz, gx))).astype(np.uint8)
+        grid[:, 0] = 1                                   # a floor
+    else:                                                # one palette entry: id 0 is "empty", so only boxes show
+        grid = np.zeros((E, gy, gz, gx), np.uint8)
+    boxes = np.zeros((E, nb, 8), np.int32)
+    count = np.full(E, nb, np.int32)
+    for e in range(E):
+        items = []
+        for _ in range(nb):
+            c = rng.uniform([1, 1, 1], [gx - 1, gy - 1, gz - 1])
+            h = rng.uniform(0.2, 1.2, 3)
+            items.append((tuple(c - h), tuple(c + h), int(rng.integers(0, P))))
+        boxes[e] = box_rows(items)
+    cams = []
+    for o in range(E * A):
+        inside = o % 3 != 2
+        pos = rng.uniform([1, 1.2, 1], [gx - 1, gy - 0.5, gz - 1]) if inside else \
+            np.array([gx / 2, gy / 2, gz / 2]) + rng.normal(0, 1, 3) * np.array([gx, gy, gz])
+        tgt = np.array([gx / 2, gy / 3, gz / 2]) + rng.normal(0, 2, 3)
+        v = tgt - pos
+        yaw = math.atan2(v[0], v[2]); pitch = math.atan2(v[1], math.hypot(v[0], v[2]))
+        cams.append(cam_row(*pos, yaw, float(np.clip(pitch, -1.3, 1.3))))
+    g_rgb, g_depth, status, st = _render_custom(oracle, grid, _pal(E, P, seed=W), np.stack(cams), W, H, boxes=boxes,
+                                                box_count=count, agents=A, max_boxes=nb, **case["kw"])
+    assert status == 0
+    parity.assert_parity(st, f"descriptor corner {W}x{H}")
+    assert st["pixels"] == E * A * W * H
+    miss = case["kw"].get("miss_depth", 0.0)
+    assert (g_depth != miss).mean() > 0.05            # something was hit
 
 
 def test_bounded_wait_runs_out_and_reports_a_status():
