@@ -419,6 +419,7 @@ def test_odd_grid_sizes_and_occupied_bounds(oracle):
     dict(W=24, H=20, grid=(20, 8, 12), P=256, kw=dict(hfov_rad=2.6, ambient=1.0, miss_depth=-1.0, sky_rgb=(0, 255, 3))),
     dict(W=136, H=68, grid=(16, 32, 16), P=7, kw=dict(hfov_rad=1.2, light_dir=(-1.0, -0.2, 0.0), miss_depth=1000.0)),
     dict(W=64, H=36, grid=(36, 12, 8), P=16, kw=dict(light_dir=(0.0, 0.0, -3.0), ambient=0.5)),
+    dict(W=512, H=288, grid=(16, 8, 16), P=16, kw=dict(hfov_rad=1.0)),       # 4608 tiles per observation
 ])
 def test_descriptor_corners(oracle, case):
     """Descriptor fields away from the workloads' defaults: smallest image, image sizes that are no
