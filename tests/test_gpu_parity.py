@@ -462,6 +462,25 @@ def test_descriptor_corners(oracle, case):
     assert (g_depth != miss).mean() > 0.05            # something was hit
 
 
+def test_longest_grid_axis_thousand_steps(oracle):
+    """The largest grid dimension the ABI takes (1024): rays that cross about a thousand cells before they
+    hit a far wall.  Crossing times are accumulated in float, so this is where the depth error is largest
+    (bounded by steps x 2^-24 relative, inside the 1e-4 bar) and where the walk's exit margin is widest."""
+    gx, gy, gz = 1024, 4, 8
+    grid = np.zeros((2, gy, gz, gx), np.uint8)
+    grid[:, 0] = 1                                  # floor
+    grid[0, :, :, 1020] = 2                         # a wall across the far end
+    grid[1, :, :, 3] = 3                            # env 1: the wall at the near end, seen from the far end
+    grid[:, 1, 4, 500] = 4                          # a lone voxel on the way, beside the view axis
+    cams = np.stack([cam_row(0.5, 2.0, 3.6, math.pi / 2, 0.0),            # looks along +x
+                     cam_row(1023.4, 2.1, 4.2, -math.pi / 2, 0.0002)])    # looks along -x
+    # a field of view so narrow that the whole image stays inside the 8 x 4 cross-section for 1000 cells
+    g_rgb, g_depth, status, st = _render_custom(oracle, grid, _pal(2, 8), cams, 64, 36, hfov_rad=0.003)
+    assert status == 0
+    parity.assert_parity(st, "1024-long grid")
+    assert (g_depth[0] > 1000).mean() > 0.3 and (g_depth[1] > 1000).mean() > 0.3     # the far walls are what is seen
+
+
 def test_bounded_wait_runs_out_and_reports_a_status():
     """Failure detection without a fault: the staging copy is withheld, every CTA's bounded wait gives
     up, the host reads a timeout status, and the same batch renders normally afterwards."""
