@@ -19,7 +19,11 @@ namespace {
 #ifndef MV_NT
 #define MV_NT 384
 #endif
-constexpr int kRenderThreads = MV_NT;
+constexpr int kRenderThreads = MV_NT;          // threads per CTA of the render kernel...
+constexpr int kRenderThreadsSmall = MV_NT / 2; // ...and for CTAs with few tiles (small images): twice as many, shorter CTAs per SM
+// Below this many tiles per CTA the small shape is faster when there are CTAs enough to fill the GPU with it
+// (measured: 64x36 images +10 %; 128x72 -2 %; four CTAs alone on the GPU -20 %: fewer warps per CTA, longer CTA).
+constexpr int kSmallCtaTiles = 192;
 constexpr int kHostChunks = 8;
 // Staging + set-up of a CTA, in units of one observation's render time, as measured on B200 at 128x72:
 // 0.15 to 0.18 for 64x16x64 grids, 0.10 for 128x32x128 grids (where a second agent's tables usually cost
@@ -58,6 +62,8 @@ struct mv_batch {
     struct Smem { uint32_t tile_off, agent_off, agent_stride, agent_ov_off, agent_mask_off, agent_ovtile_off, misc_off, bytes; };
     Smem smem{};                        // shared-memory layout of the render kernel for agents_per_cta
     int agents_per_cta = 1;             // observations one CTA renders: 1, or every agent of its env
+    int threads = MV_NT;                // threads per CTA of the render kernel (fewer for CTAs with few tiles)
+    int sms = 0;
     int tiles_x = 0, tiles_y = 0, mask_words = 0;
     int64_t launches = 0;
     int wait_polls = 1 << 18;
@@ -128,10 +134,22 @@ mv_batch::Smem smem_layout(const mv_batch *b, int apc) {
     return m;
 }
 
+// Threads per CTA: the small shape for CTAs with few tiles, if the batch has CTAs enough to fill the GPU
+// six to an SM.
+int pick_threads(const mv_batch *b, int apc) {
+    const bool few_tiles = b->tiles_x * b->tiles_y * apc < kSmallCtaTiles;
+    const bool fills = (int64_t)b->num_obs / apc >= (int64_t)6 * b->sms;
+    return few_tiles && fills ? kRenderThreadsSmall : kRenderThreads;
+}
+
 // The three instantiations of the render kernel: column-word walk (grid at most 32 high, occupancy
 // staged), indexed walk with staged occupancy, indexed walk with the occupancy in global memory.
 using RenderFn = void (*)(const RenderParams);
 RenderFn render_fn(const mv_batch *b) {
+    if (b->threads == kRenderThreadsSmall) {
+        if (!b->occ_shared) return render_kernel<kRenderThreadsSmall, false, false>;
+        return b->lay.ysh == 5 ? render_kernel<kRenderThreadsSmall, true, true> : render_kernel<kRenderThreadsSmall, true, false>;
+    }
     if (!b->occ_shared) return render_kernel<kRenderThreads, false, false>;
     return b->lay.ysh == 5 ? render_kernel<kRenderThreads, true, true> : render_kernel<kRenderThreads, true, false>;
 }
@@ -170,7 +188,7 @@ int launch_render(mv_batch *b, uint8_t *d_rgb, float *d_depth, int obs_begin, in
     p.wait_polls = b->wait_polls;
     p.skip_staging = b->skip_staging;
     const int ctas = obs_count / b->agents_per_cta;   // callers pass whole environments when a CTA renders one
-    render_fn(b)<<<ctas, kRenderThreads, b->smem.bytes - unstaged, s>>>(p);
+    render_fn(b)<<<ctas, b->threads, b->smem.bytes - unstaged, s>>>(p);
     b->launches++;
     MV_CUDA(b, cudaGetLastError());
     return MV_OK;
@@ -409,7 +427,9 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
     // The dynamic shared-memory cap is a property of the kernel function on this device, shared by
     // every batch: raise it to the device's maximum once, never to one batch's own size.
     for (RenderFn f : {RenderFn(render_kernel<kRenderThreads, true, true>), RenderFn(render_kernel<kRenderThreads, true, false>),
-                       RenderFn(render_kernel<kRenderThreads, false, false>)})
+                       RenderFn(render_kernel<kRenderThreads, false, false>), RenderFn(render_kernel<kRenderThreadsSmall, true, true>),
+                       RenderFn(render_kernel<kRenderThreadsSmall, true, false>),
+                       RenderFn(render_kernel<kRenderThreadsSmall, false, false>)})
         if (e == cudaSuccess) e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max);
     if (e != cudaSuccess) { delete b; return MV_ERR_CUDA; }
     // One CTA per environment (block staged once for all its agents) when that still fills the GPU;
@@ -432,6 +452,9 @@ int mv_create_batch(const mv_batch_desc *desc, mv_batch **out) {
             }
         }
     }
+
+    b->sms = sms;
+    b->threads = pick_threads(b, b->agents_per_cta);
 
     const size_t blocks_bytes = (size_t)d.num_envs * L.stride;
     bool ok = cudaMalloc(&b->d_env_blocks, blocks_bytes) == cudaSuccess &&
@@ -671,6 +694,7 @@ int mv_debug_agents_per_cta(mv_batch *b, int agents_per_cta) {
     if (!b->occ_fits_shared) b->occ_shared = false;
     b->smem = m;
     b->agents_per_cta = apc;
+    b->threads = pick_threads(b, apc);
     return MV_OK;
 }
 

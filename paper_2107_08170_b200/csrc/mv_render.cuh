@@ -207,7 +207,7 @@ __device__ __forceinline__ void write_sky(uint8_t *rgb_obs, float *depth_obs, in
 // occupancy is read from global memory through the read-only path.
 // COLW: column-word flavour of the walk (grid at most 32 high and occupancy staged).
 template <int NT, bool OCC_SHARED, bool COLW>
-__global__ void __launch_bounds__(NT, MV_MINB) render_kernel(const RenderParams p)
+__global__ void __launch_bounds__(NT, (MV_MINB * 384) / NT) render_kernel(const RenderParams p)
 {
     static_assert(OCC_SHARED || !COLW, "the column-word walk reads shared memory");
     extern __shared__ __align__(128) unsigned char smem[];
