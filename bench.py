@@ -35,9 +35,9 @@ WORKLOAD = "headline"
 # capture of render_kernel on a 2048-environment slice of the headline workload (summary and command in
 # profiles/render_kernel_headline_2048env_ncu_full.md); NCU_BUILD names the commit of the library they were
 # taken on.  DRAM traffic grows in proportion to the environments, so a full launch is the slice x 8.
-NCU_BUILD = "be3d5f8"
+NCU_BUILD = "4762628"
 NCU_SLICE_ENVS = 2048
-NCU_SLICE_DRAM_BYTES = 147.44e6 + 84.28e6   # dram__bytes_read.sum + dram__bytes_write.sum of one launch on the slice
+NCU_SLICE_DRAM_BYTES = 147.42e6 + 85.17e6   # dram__bytes_read.sum + dram__bytes_write.sum of one launch on the slice
 NCU_WARP_INSTRUCTIONS_PER_TILE = 233.9  # smsp__inst_executed.sum / (8x4-pixel tiles) on the slice
 
 
